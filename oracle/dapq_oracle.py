@@ -1,0 +1,190 @@
+"""CPU oracle for the DapQ eviction scorer.  TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+
+A plain, slow, float64 numpy statement of what the scorer computes, written from
+the paper's definitions so that it can be checked against them by eye.  It shares
+no code with the CUDA library and is imported only by the tests, the smoke check
+and the benchmark's CPU-baseline leg.
+
+Every function is pinned by the CPU tests (library causal attention on tiny
+inputs, closed forms, invariants, equivariances, hand-worked cases): no function
+here is "parity unpinned".
+
+Notation (paper, Section 4): L_p prompt length, N pseudo tokens placed at
+positions L_p .. L_p+N-1, d_k head dimension, S(j) importance of prompt token j,
+K the number of retained tokens.  G is the number of query heads that share one
+KV head (grouped-query attention; the paper's models are GQA, its equations carry
+no head index, so scores of a group are summed: Eq. 4 is a sum).
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.1: pseudo queries carry the positional encodings of positions L_p .. L_p+N-1
+# --------------------------------------------------------------------------------------
+def rope_inv_freq(head_dim: int, rope_base: float) -> np.ndarray:
+    """theta_c = base^(-2c/d), c = 0 .. d/2-1 (rotary position embedding frequencies)."""
+    c = np.arange(head_dim // 2, dtype=np.float64)
+    return np.power(np.float64(rope_base), -2.0 * c / np.float64(head_dim))
+
+
+def rope_pseudo_q(q_pre: np.ndarray, pos_start: int, rope_base: float,
+                  inv_freq: Optional[np.ndarray] = None) -> np.ndarray:
+    """Rotate pseudo queries to positions pos_start + i (Section 4.1, position assignment).
+
+    q_pre [..., N, d].  Rotate-half pairing: channel c is paired with channel c + d/2,
+      out[c]       = q[c]     cos(p theta_c) - q[c+d/2] sin(p theta_c)
+      out[c + d/2] = q[c+d/2] cos(p theta_c) + q[c]     sin(p theta_c).
+    """
+    q = np.asarray(q_pre, dtype=np.float64)
+    n, d = q.shape[-2], q.shape[-1]
+    half = d // 2
+    theta = rope_inv_freq(d, rope_base) if inv_freq is None else np.asarray(inv_freq, np.float64)
+    pos = np.float64(pos_start) + np.arange(n, dtype=np.float64)
+    ang = pos[:, None] * theta[None, :]                    # [N, d/2]
+    cos, sin = np.cos(ang), np.sin(ang)
+    lo, hi = q[..., :half], q[..., half:]
+    out = np.empty_like(q)
+    out[..., :half] = lo * cos - hi * sin
+    out[..., half:] = hi * cos + lo * sin
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.2, Eq. 4: S(j) = sum_i Attention(q_i, k_j),  Attention = softmax(q K^T / sqrt(d_k))
+# --------------------------------------------------------------------------------------
+def visible_logits(q_rot_h: np.ndarray, keys: np.ndarray, prompt_len: int,
+                   scale: Optional[float] = None) -> np.ndarray:
+    """Pre-softmax scores s_ij = q_i . k_j / sqrt(d_k) with unseen keys set to -inf.
+
+    q_rot_h [N, d]; keys [L_p + N, d]: L_p prompt keys followed by the N synthetic
+    keys.  Pseudo query i sits at position L_p + i, so under the causal mask of the
+    extended prefill it sees every prompt key and synthetic keys 0 .. i (itself
+    included).  (Appendix C, Step 1 for s_j; Section 6.3 for the causal mask.)
+    """
+    q = np.asarray(q_rot_h, dtype=np.float64)
+    kk = np.asarray(keys, dtype=np.float64)
+    n, d = q.shape
+    L = int(prompt_len)
+    assert kk.shape[0] == L + n
+    sc = 1.0 / math.sqrt(d) if scale is None else float(scale)
+    s = (q @ kk.T) * sc                                      # [N, L+N]
+    col = np.arange(L + n)[None, :]
+    row = np.arange(n)[:, None]
+    visible = (col < L) | ((col - L) <= row)
+    return np.where(visible, s, -np.inf)
+
+
+def attention_rows(q_rot_h: np.ndarray, keys: np.ndarray, prompt_len: int,
+                   scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention weights of one head's N pseudo queries, and their log-sum-exp.
+
+    Returns P [N, L_p + N], each row softmax(s) over the visible span (masked entries
+    exactly 0; weights >= 0 and summing to 1), and lse [N] = log sum_j exp(s_ij).
+    """
+    s = visible_logits(q_rot_h, keys, prompt_len, scale)
+    m = s.max(axis=1, keepdims=True)
+    e = np.exp(s - m)
+    z = e.sum(axis=1, keepdims=True)
+    return e / z, (m + np.log(z))[:, 0]
+
+
+def score_sequence(q_rot: np.ndarray, k_seq: np.ndarray, prompt_len: int, group: int,
+                   scale: Optional[float] = None) -> Dict[str, np.ndarray]:
+    """Importance scores of one sequence's prompt tokens, per KV head (Eq. 4 + GQA sum).
+
+    q_rot [H_q, N, d] rotated pseudo queries; k_seq [H_kv, L_p + N, d] that sequence's
+    keys (prompt rows then synthetic rows).  Query head h reads KV head h // G.
+    Returns
+      scores      [H_kv, L_p]  sum over the group's G heads and the N queries of P_ij
+      lse         [H_q, N]     log sum_j exp(s_ij) over the visible span
+      prompt_mass [H_q]        sum_i sum_{j < L_p} P_ij
+      syn_mass    [H_q]        sum_i sum_{synthetic j} P_ij   (prompt + syn = N)
+    """
+    q = np.asarray(q_rot, dtype=np.float64)
+    Hq, n, d = q.shape
+    Hkv = k_seq.shape[0]
+    L = int(prompt_len)
+    assert Hq == Hkv * group
+    scores = np.zeros((Hkv, L), dtype=np.float64)
+    lse = np.zeros((Hq, n), dtype=np.float64)
+    pm = np.zeros(Hq, dtype=np.float64)
+    sm = np.zeros(Hq, dtype=np.float64)
+    for h in range(Hq):
+        kv = h // group
+        P, lse[h] = attention_rows(q[h], k_seq[kv], L, scale)
+        S_h = P[:, :L].sum(axis=0)                           # Eq. 4: sum over the N queries
+        scores[kv] += S_h                                    # GQA: sum over the group
+        pm[h] = S_h.sum()
+        sm[h] = P[:, L:].sum()
+    return {"scores": scores, "lse": lse, "prompt_mass": pm, "syn_mass": sm}
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.2, Eq. 5: M_retain = TopK_j S(j)
+# --------------------------------------------------------------------------------------
+def topk_select(scores: np.ndarray, k_keep: int) -> np.ndarray:
+    """Indices of the k_keep largest scores, returned in ascending position order.
+
+    Full sort on (score descending, index ascending): ties at the threshold go to
+    the lower index.  k_keep larger than the length keeps everything.
+    """
+    s = np.asarray(scores, dtype=np.float64)
+    L = s.shape[0]
+    kk = min(int(k_keep), L)
+    order = np.lexsort((np.arange(L), -s))                   # last key is the primary one
+    return np.sort(order[:kk]).astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.2, last paragraph: prune the cache to M_retain, drop every synthetic token
+# --------------------------------------------------------------------------------------
+def compact_kv(k_seq_head: np.ndarray, v_seq_head: np.ndarray,
+               idx: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Rows idx of one head's K and V, copied unchanged (same rows for K and V)."""
+    return k_seq_head[idx].copy(), v_seq_head[idx].copy()
+
+
+def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int],
+          prompt_len: Sequence[int], k_keep: Sequence[int], rope_base: float,
+          scale: Optional[float] = None,
+          pos_start: Optional[Sequence[int]] = None) -> Dict[str, object]:
+    """The whole path for one layer (Figure 1): rotate, score, select, compact.
+
+    q_pre [B, H_q, N, d] pre-RoPE pseudo queries (any float dtype; converted exactly
+    to float64); k, v [H_kv, R, d] packed cache whose sequence b owns rows
+    cu_rows[b] .. cu_rows[b+1] (L_b prompt rows, then N synthetic rows).
+    Returns per-sequence lists: scores [H_kv, L_b], idx [H_kv, K_b] (sequence-local),
+    k_out / v_out [H_kv, K_b, d] in the dtype of k / v, plus lse and the two masses.
+    """
+    B, Hq, n, d = q_pre.shape
+    Hkv = k.shape[0]
+    G = Hq // Hkv
+    out: Dict[str, List] = {key: [] for key in
+                            ("q_rot", "scores", "lse", "prompt_mass", "syn_mass",
+                             "idx", "k_out", "v_out")}
+    for b in range(B):
+        L = int(prompt_len[b])
+        r0 = int(cu_rows[b])
+        assert int(cu_rows[b + 1]) - r0 == L + n
+        p0 = L if pos_start is None else int(pos_start[b])
+        q_rot = rope_pseudo_q(np.asarray(q_pre[b], dtype=np.float64), p0, rope_base)
+        k_seq = k[:, r0:r0 + L + n]
+        v_seq = v[:, r0:r0 + L + n]
+        res = score_sequence(q_rot, k_seq, L, G, scale)
+        kk = min(int(k_keep[b]), L)
+        idx = np.stack([topk_select(res["scores"][h], kk) for h in range(Hkv)])
+        kept = [compact_kv(k_seq[h], v_seq[h], idx[h]) for h in range(Hkv)]
+        ko = np.stack([kv[0] for kv in kept])
+        vo = np.stack([kv[1] for kv in kept])
+        out["q_rot"].append(q_rot)
+        for key in ("scores", "lse", "prompt_mass", "syn_mass"):
+            out[key].append(res[key])
+        out["idx"].append(idx)
+        out["k_out"].append(ko)
+        out["v_out"].append(vo)
+    return out

@@ -1,0 +1,307 @@
+"""CPU pins for the oracle: every oracle function is checked against something other
+than itself - a library routine, a closed form, an invariant, a hand-worked case or
+brute force on tiny inputs - before any CUDA result is compared with it."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dapq_oracle as orc
+
+
+def _rand(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape)
+
+
+# ------------------------------------------------------------------ RoPE (Section 4.1)
+def test_rope_quarter_and_half_turns():
+    # Plane rotations by 90 and 180 degrees have exact images: pair (1,3) -> (-3,1),
+    # pair (2,4) -> (-2,-4).  Pairs are (c, c + d/2).
+    q = np.array([[1.0, 2.0, 3.0, 4.0]])
+    out = orc.rope_pseudo_q(q, pos_start=1, rope_base=1.0,
+                            inv_freq=np.array([math.pi / 2, math.pi]))
+    np.testing.assert_allclose(out, [[-3.0, -2.0, 1.0, -4.0]], atol=1e-14)
+
+
+def test_rope_positions_advance_by_one_per_pseudo_query():
+    # Query i sits at pos_start + i: with theta = pi/2 and q = e_0 the four queries
+    # at positions 4,5,6,7 point along +x, +y, -x, -y of the (0, 1) pair.
+    q = np.tile(np.array([[1.0, 0.0]]), (4, 1))
+    out = orc.rope_pseudo_q(q, pos_start=4, rope_base=1.0, inv_freq=np.array([math.pi / 2]))
+    np.testing.assert_allclose(out, [[1, 0], [0, 1], [-1, 0], [0, -1]], atol=1e-14)
+
+
+def test_rope_inv_freq_closed_form():
+    # base^(-2c/d): for d = 8, base = 10^4 the frequencies are 1, 0.1, 0.01, 0.001.
+    np.testing.assert_allclose(orc.rope_inv_freq(8, 1.0e4), [1.0, 0.1, 0.01, 0.001], rtol=1e-14)
+
+
+def test_rope_matches_transformers_llama():
+    tf = pytest.importorskip("transformers.models.llama.modeling_llama")
+    from transformers import LlamaConfig
+    d, n, pos0 = 16, 5, 37
+    cfg = LlamaConfig(hidden_size=4 * d, num_attention_heads=4, head_dim=d, rope_theta=5.0e5)
+    rot = tf.LlamaRotaryEmbedding(cfg)
+    q = _rand((1, 4, n, d), 1)
+    qt = torch.from_numpy(q)
+    cos, sin = rot(qt, torch.arange(pos0, pos0 + n)[None])
+    lib, _ = tf.apply_rotary_pos_emb(qt, qt, cos.double(), sin.double())
+    mine = orc.rope_pseudo_q(q[0], pos0, 5.0e5)
+    # the library builds its table in float32
+    np.testing.assert_allclose(mine, lib[0].numpy(), atol=2e-5)
+
+
+def test_rope_identity_norm_and_relative_property():
+    q, k = _rand((3, 6, 32), 2), _rand((3, 6, 32), 3)
+    np.testing.assert_array_equal(orc.rope_pseudo_q(q[:, :1], 0, 1.0e4), q[:, :1])
+    r = orc.rope_pseudo_q(q, 1000, 1.0e4)
+    np.testing.assert_allclose(np.linalg.norm(r, axis=-1), np.linalg.norm(q, axis=-1), rtol=1e-13)
+    # <R_m q, R_n k> depends on m - n only
+    for shift in (1, 77, 4096):
+        a = np.einsum("hnd,hnd->hn", orc.rope_pseudo_q(q, 50, 1.0e4), orc.rope_pseudo_q(k, 20, 1.0e4))
+        b = np.einsum("hnd,hnd->hn", orc.rope_pseudo_q(q, 50 + shift, 1.0e4),
+                      orc.rope_pseudo_q(k, 20 + shift, 1.0e4))
+        np.testing.assert_allclose(a, b, atol=1e-9)
+
+
+def test_rope_angle_precision_at_128k():
+    # double-precision angles at the largest position used (131072 + 127) agree with
+    # extended precision to far below the scorer's tolerance
+    d, base, pos = 128, 5.0e5, 131072 + 127
+    c = np.arange(d // 2, dtype=np.longdouble)
+    theta = np.power(np.longdouble(base), -2 * c / np.longdouble(d))
+    ang = np.longdouble(pos) * theta
+    q = np.ones((1, d))
+    out = orc.rope_pseudo_q(q, pos, base)[0]
+    ref_lo = (np.cos(ang) - np.sin(ang)).astype(np.float64)
+    ref_hi = (np.cos(ang) + np.sin(ang)).astype(np.float64)
+    np.testing.assert_allclose(out[:d // 2], ref_lo, atol=1e-9)
+    np.testing.assert_allclose(out[d // 2:], ref_hi, atol=1e-9)
+
+
+# ------------------------------------------------ scorer (Eq. 4) vs library causal attention
+def sdpa_scores(q_rot, k_seq, L, G, scale=None):
+    """Column sums from textbook causal attention over the whole extended sequence.
+
+    torch's scaled_dot_product_attention with V = identity returns the attention
+    matrix itself; rows L.. are the pseudo queries (rows < L carry arbitrary
+    queries, their outputs are ignored)."""
+    Hq, n, d = q_rot.shape
+    Hkv = k_seq.shape[0]
+    T = L + n
+    out = np.zeros((Hkv, L))
+    eye = torch.eye(T, dtype=torch.float64)[None, None]
+    for h in range(Hq):
+        qfull = np.concatenate([_rand((L, d), 100 + h), q_rot[h]], axis=0)
+        P = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(qfull)[None, None], torch.from_numpy(np.ascontiguousarray(k_seq[h // G]))[None, None],
+            eye, is_causal=True, scale=scale)[0, 0].numpy()
+        out[h // G] += P[L:, :L].sum(axis=0)
+    return out
+
+
+@pytest.mark.parametrize("L,n,d,Hkv,G", [(1, 1, 4, 1, 1), (5, 3, 8, 2, 2), (17, 3, 128, 1, 4),
+                                         (64, 8, 16, 2, 1), (33, 7, 32, 3, 3)])
+def test_score_equals_library_causal_attention(L, n, d, Hkv, G):
+    q = _rand((Hkv * G, n, d), 5)
+    k = _rand((Hkv, L + n, d), 6)
+    got = orc.score_sequence(q, k, L, G)["scores"]
+    np.testing.assert_allclose(got, sdpa_scores(q, k, L, G), rtol=1e-11, atol=1e-14)
+
+
+def test_score_custom_scale_matches_library():
+    q, k = _rand((2, 3, 8), 7), _rand((1, 9 + 3, 8), 8)
+    got = orc.score_sequence(q, k, 9, 2, scale=0.7)["scores"]
+    np.testing.assert_allclose(got, sdpa_scores(q, k, 9, 2, scale=0.7), rtol=1e-11)
+
+
+def test_pins_catch_planted_mistakes(monkeypatch):
+    """The library pin must fail for plausible mistakes in the oracle (planted here)."""
+    q, k = _rand((4, 3, 8), 9), _rand((2, 12 + 3, 8), 10)
+    ref = sdpa_scores(q, k, 12, 2)
+    good = orc.visible_logits
+
+    def strict_causal(qh, keys, L, scale=None):          # self not visible
+        s = good(qh, keys, L, scale).copy()
+        n = qh.shape[0]
+        for i in range(1, n):
+            s[i, L + i] = -np.inf
+        return s
+
+    def no_scale(qh, keys, L, scale=None):               # dropped 1/sqrt(d)
+        return good(qh, keys, L, 1.0)
+
+    def prompt_only(qh, keys, L, scale=None):            # synthetic keys left out of the span
+        s = good(qh, keys, L, scale).copy()
+        s[:, L + 1:] = -np.inf
+        return s
+
+    for bad in (strict_causal, no_scale, prompt_only):
+        monkeypatch.setattr(orc, "visible_logits", bad)
+        got = orc.score_sequence(q, k, 12, 2)["scores"]
+        assert not np.allclose(got, ref, rtol=1e-6), bad.__name__
+    monkeypatch.setattr(orc, "visible_logits", good)
+    # wrong head -> KV head map (interleaved instead of blocked groups)
+    got = orc.score_sequence(q[[0, 2, 1, 3]], k, 12, 2)["scores"]
+    assert not np.allclose(got, ref, rtol=1e-6)
+    np.testing.assert_allclose(orc.score_sequence(q, k, 12, 2)["scores"], ref, rtol=1e-11)
+
+
+# ------------------------------------------------------------------------- closed forms
+def test_identical_keys_give_harmonic_scores():
+    # all keys equal -> every row is uniform over its L + i + 1 visible keys
+    L, n, d = 11, 6, 8
+    k = np.tile(_rand((1, 1, d), 11), (1, L + n, 1))
+    q = _rand((1, n, d), 12)
+    res = orc.score_sequence(q, k, L, 1)
+    expect = sum(1.0 / (L + i + 1) for i in range(n))
+    np.testing.assert_allclose(res["scores"][0], np.full(L, expect), rtol=1e-13)
+    np.testing.assert_allclose(res["lse"][0], [math.log(L + i + 1) + float(q[0, i] @ k[0, 0]) / math.sqrt(d)
+                                               for i in range(n)], rtol=1e-12)
+
+
+def test_single_query_single_head_is_one_softmax_row():
+    scipy_special = pytest.importorskip("scipy.special")
+    L, d = 23, 16
+    q, k = _rand((1, 1, d), 13), _rand((1, L + 1, d), 14)
+    row = scipy_special.softmax((k[0] @ q[0, 0]) / math.sqrt(d))
+    res = orc.score_sequence(q, k, L, 1)
+    np.testing.assert_allclose(res["scores"][0], row[:L], rtol=1e-12)
+    np.testing.assert_allclose(res["syn_mass"][0], row[L], rtol=1e-12)
+    np.testing.assert_allclose(res["lse"][0, 0], scipy_special.logsumexp((k[0] @ q[0, 0]) / math.sqrt(d)),
+                               rtol=1e-13)
+
+
+# --------------------------------------------------------------------------- invariants
+def test_rows_sum_to_one_and_mass_is_conserved():
+    L, n, d, Hkv, G = 300, 16, 64, 2, 4
+    q, k = _rand((Hkv * G, n, d), 15) * 2.0, _rand((Hkv, L + n, d), 16) * 2.0
+    for h in range(Hkv * G):
+        P, _ = orc.attention_rows(q[h], k[h // G], L)
+        assert (P >= 0).all()
+        np.testing.assert_allclose(P.sum(axis=1), np.ones(n), rtol=1e-12)
+        # causal span: query i never sees synthetic key i' > i
+        assert np.all(np.triu(P[:, L:], k=1) == 0.0) and np.all(np.diagonal(P[:, L:]) > 0)
+    res = orc.score_sequence(q, k, L, G)
+    np.testing.assert_allclose(res["prompt_mass"] + res["syn_mass"], np.full(Hkv * G, n), rtol=1e-12)
+    np.testing.assert_allclose(res["scores"].sum(axis=1) + res["syn_mass"].reshape(Hkv, G).sum(axis=1),
+                               np.full(Hkv, G * n), rtol=1e-12)
+
+
+def test_equivariances():
+    L, n, d, Hkv, G = 40, 5, 16, 2, 3
+    q, k = _rand((Hkv * G, n, d), 17), _rand((Hkv, L + n, d), 18)
+    base = orc.score_sequence(q, k, L, G)["scores"]
+    # permuting heads inside a group changes nothing; swapping groups swaps KV heads
+    perm = np.array([2, 0, 1, 4, 5, 3])
+    np.testing.assert_allclose(orc.score_sequence(q[perm], k, L, G)["scores"], base, rtol=1e-12)
+    swap = np.array([3, 4, 5, 0, 1, 2])
+    np.testing.assert_allclose(orc.score_sequence(q[swap], k[::-1], L, G)["scores"], base[::-1], rtol=1e-12)
+    # permuting prompt rows (keys are stored post-RoPE) permutes the scores
+    p = np.random.default_rng(19).permutation(L)
+    kp = k.copy()
+    kp[:, :L] = k[:, p]
+    np.testing.assert_allclose(orc.score_sequence(q, kp, L, G)["scores"], base[:, p], rtol=1e-12)
+    # adding one vector to every key shifts each row's logits by a constant
+    shift = _rand((d,), 20)
+    np.testing.assert_allclose(orc.score_sequence(q, k + shift, L, G)["scores"], base, rtol=1e-10)
+
+
+def test_theorem_bounds_hold():
+    # Appendix C, inequalities (4) and (5): for unit q, q' the largest logit gap and the
+    # L1 gap of the attention rows are bounded by K_max * |q - q'| / sqrt(d_k)
+    rng = np.random.default_rng(21)
+    d, L = 32, 200
+    k = rng.standard_normal((1, L + 1, d))
+    kmax = np.linalg.norm(k[0], axis=1).max()
+    for _ in range(20):
+        q = rng.standard_normal(d)
+        q /= np.linalg.norm(q)
+        q2 = q + 0.3 * rng.standard_normal(d)
+        q2 /= np.linalg.norm(q2)
+        bound = kmax * math.sqrt(2 * (1 - float(q @ q2))) / math.sqrt(d)
+        a, _ = orc.attention_rows(q[None], k[0], L)
+        b, _ = orc.attention_rows(q2[None], k[0], L)
+        sa = orc.visible_logits(q[None], k[0], L)
+        sb = orc.visible_logits(q2[None], k[0], L)
+        assert np.abs(sa - sb).max() <= bound + 1e-12
+        assert np.abs(a - b).sum() <= bound + 1e-12
+
+
+# ------------------------------------------------------------------- top-K (Eq. 5)
+def test_topk_hand_cases():
+    s = np.array([0.5, 0.2, 0.5, 0.1, 0.2])
+    np.testing.assert_array_equal(orc.topk_select(s, 1), [0])          # tie -> lower index
+    np.testing.assert_array_equal(orc.topk_select(s, 2), [0, 2])
+    np.testing.assert_array_equal(orc.topk_select(s, 3), [0, 1, 2])    # tie at threshold -> index 1
+    np.testing.assert_array_equal(orc.topk_select(s, 4), [0, 1, 2, 4])
+    np.testing.assert_array_equal(orc.topk_select(s, 5), [0, 1, 2, 3, 4])
+    np.testing.assert_array_equal(orc.topk_select(s, 9), [0, 1, 2, 3, 4])  # clamp
+    np.testing.assert_array_equal(orc.topk_select(np.zeros(4), 2), [0, 1])
+    assert orc.topk_select(s, 3).dtype == np.int32
+
+
+def test_topk_properties_and_library_agreement():
+    rng = np.random.default_rng(22)
+    for L, K in [(1, 1), (100, 7), (1000, 999), (4097, 128)]:
+        s = rng.random(L)
+        idx = orc.topk_select(s, K)
+        assert len(idx) == K and np.all(np.diff(idx) > 0) and idx.min() >= 0 and idx.max() < L
+        rest = np.setdiff1d(np.arange(L), idx)
+        assert rest.size == 0 or s[idx].min() >= s[rest].max()
+        lib = torch.topk(torch.from_numpy(s), K).indices.numpy()      # distinct values: unique set
+        np.testing.assert_array_equal(idx, np.sort(lib))
+
+
+# --------------------------------------------------------------- compaction / full path
+def test_compaction_is_a_bit_exact_row_copy_without_synthetic_rows():
+    rng = np.random.default_rng(23)
+    B, Hq, Hkv, n, d = 2, 4, 2, 3, 8
+    Ls, Ks = [19, 7], [5, 9]
+    cu = np.concatenate([[0], np.cumsum([l + n for l in Ls])])
+    q = rng.standard_normal((B, Hq, n, d))
+    k = rng.standard_normal((Hkv, cu[-1], d)).astype(np.float32)
+    v = rng.standard_normal((Hkv, cu[-1], d)).astype(np.float32)
+    res = orc.evict(q, k, v, cu, Ls, Ks, 1.0e4)
+    for b in range(B):
+        idx = res["idx"][b]
+        kk = min(Ks[b], Ls[b])
+        assert idx.shape == (Hkv, kk) and idx.max() < Ls[b]          # never a synthetic row
+        for h in range(Hkv):
+            assert res["k_out"][b][h].tobytes() == k[h, cu[b] + idx[h]].tobytes()
+            assert res["v_out"][b][h].tobytes() == v[h, cu[b] + idx[h]].tobytes()
+            assert res["k_out"][b].dtype == np.float32
+    # K_b >= L_b keeps every prompt row, in order
+    np.testing.assert_array_equal(res["idx"][1][0], np.arange(7))
+
+
+def test_evict_uses_decode_positions():
+    # the path rotates sequence b's queries to L_b .. L_b+N-1 (Section 4.1)
+    rng = np.random.default_rng(24)
+    q = rng.standard_normal((1, 2, 4, 16))
+    k = rng.standard_normal((1, 30 + 4, 16))
+    res = orc.evict(q, k, k, [0, 34], [30], [5], 1.0e4)
+    np.testing.assert_array_equal(res["q_rot"][0], orc.rope_pseudo_q(q[0], 30, 1.0e4))
+    direct = orc.score_sequence(orc.rope_pseudo_q(q[0], 30, 1.0e4), k, 30, 2)["scores"]
+    np.testing.assert_array_equal(res["scores"][0], direct)
+    other = orc.evict(q, k, k, [0, 34], [30], [5], 1.0e4, pos_start=[31])
+    assert not np.allclose(other["scores"][0], direct)
+
+
+def test_planted_needles_are_retained():
+    from gen import inputs as gi
+    w = gi.workload("tiny")
+    data = gi.draw_layer(w, 0, "cpu")
+    q_rot = np.stack([orc.rope_pseudo_q(data["q_pre"][b].double().numpy(), w.prompt_lens[b], w.rope_base)
+                      for b in range(w.batch)])
+    gi.plant_structure(w, data, torch.from_numpy(q_rot))
+    res = orc.evict(data["q_pre"].double().numpy(), data["k"].double().numpy(), data["v"].double().numpy(),
+                    w.cu_rows, w.prompt_lens, w.keep, w.rope_base)
+    for h in range(w.n_kv_heads):
+        idx = set(res["idx"][0][h].tolist())
+        sc = res["scores"][0][h]
+        kth = np.sort(sc)[-w.keep[0]]
+        for p in data["needle_pos"][0, h]:
+            assert int(p) in idx
+            assert sc[p] >= 10 * kth
