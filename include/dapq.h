@@ -1,0 +1,177 @@
+/*
+ * dapq.h - C ABI of the DapQ eviction scorer for NVIDIA B200 (sm_100a).
+ *
+ * DapQ (decoding-aligned KV cache compression via position-aware pseudo queries)
+ * appends N synthetic tokens to a prompt of length L_p, gives them the positions
+ * L_p .. L_p+N-1 of the first N decoding steps, and uses their queries as the
+ * observation window that decides which prompt tokens stay in the KV cache.
+ * This library is the step that runs after the extended prefill of one layer:
+ *
+ *   1. dapq_rope_pseudo_q  rotate the pseudo queries to their decode positions
+ *                          (Section 4.1, "Positions(T_pseudo) = [L_p, ..., L_p+N-1]").
+ *   2. dapq_score          S(j) = sum_i Attention(q_i, k_j)            (Section 4.2, Eq. 4)
+ *                          with Attention = softmax(q K^T / sqrt(d_k)) (Appendix C, Theorem),
+ *                          summed over the query heads of a GQA group.
+ *   3. dapq_topk_select    M_retain = TopK_j S(j)                       (Section 4.2, Eq. 5)
+ *   4. dapq_compact_kv     keep the K/V rows in M_retain, drop the rest and every
+ *                          synthetic token (Section 4.2, last paragraph; Figure 1).
+ *   5. dapq_evict          1-4 for one layer's cache on one stream.
+ *
+ * Conventions
+ *   - One process drives one GPU.  All kernels are asynchronous on the caller's
+ *     stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - "device" pointers are caller-owned device memory that must stay valid until
+ *     the stream work finishes; "host" pointers are read before the call returns.
+ *   - The library allocates device memory only inside dapq_create (workspace sized
+ *     from dapq_shape) and, on first use, inside dapq_evict_host (staging buffers).
+ *   - Argument errors are returned synchronously and launch nothing.  A bounded
+ *     device-side wait that gives up sets a status word that dapq_poll_status reads.
+ *   - Outputs must not alias inputs.
+ *
+ * Layouts (d = head_dim = 128, G = n_q_heads / n_kv_heads, query head h reads KV head h / G)
+ *   q_pre, q_rot  [B, H_q, N, d]   contiguous, element type = dapq_shape.dtype
+ *   K, V cache    [H_kv, R, d]     strided view (strides in elements, d contiguous); the R rows
+ *                                  are packed by sequence: sequence b owns rows
+ *                                  cu_rows[b] .. cu_rows[b+1]-1 = L_b prompt rows followed by
+ *                                  its N synthetic rows.  Keys are stored already rotated.
+ *   scores        [H_kv, T]        fp32, T = sum_b L_b, sequence b at columns cu_prompt[b] ..
+ *   idx           [H_kv, KT]       int32, KT = sum_b min(K_b, L_b); sequence-local prompt
+ *                                  positions in [0, L_b), ascending within a sequence
+ *   k_out, v_out  [H_kv, KT, d]    contiguous, same element type as the cache
+ */
+#ifndef DAPQ_H
+#define DAPQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define DAPQ_API __attribute__((visibility("default")))
+#else
+#define DAPQ_API
+#endif
+
+typedef enum {
+  DAPQ_OK = 0,
+  DAPQ_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, inconsistent offsets */
+  DAPQ_ERR_UNSUPPORTED = 2,   /* head_dim != 128, N > 128, misaligned strides, ... */
+  DAPQ_ERR_WORKSPACE = 3,     /* call exceeds the sizes given to dapq_create */
+  DAPQ_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed (see dapq_last_error) */
+  DAPQ_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (dapq_poll_status) */
+} dapq_status;
+
+typedef enum { DAPQ_BF16 = 0, DAPQ_F32 = 1 } dapq_dtype;
+
+enum { DAPQ_MAX_BATCH = 128, DAPQ_MAX_PSEUDO = 128, DAPQ_HEAD_DIM = 128 };
+
+/* Pooling of the accumulated scores before selection.  The paper specifies none for
+ * DapQ (it mentions pooling only for the SnapKV / PyramidKV baselines), so NONE is the
+ * default; MAX / AVG apply a 1-D window of odd width pool_kernel, stride 1, clipped at
+ * the ends of each sequence. */
+typedef enum { DAPQ_POOL_NONE = 0, DAPQ_POOL_MAX = 1, DAPQ_POOL_AVG = 2 } dapq_pool_mode;
+
+typedef struct dapq_ctx dapq_ctx;
+
+typedef struct {
+  int32_t n_q_heads;        /* H_q                                               */
+  int32_t n_kv_heads;       /* H_kv, divides H_q                                 */
+  int32_t head_dim;         /* must be 128                                        */
+  int32_t n_pseudo;         /* N, 1 .. 128                                        */
+  int32_t max_batch;        /* largest B of any call, 1 .. DAPQ_MAX_BATCH         */
+  int32_t dtype;            /* dapq_dtype of q, K and V                           */
+  int64_t max_total_rows;   /* largest R = sum_b (L_b + N) of any call            */
+  double  rope_base;        /* theta_c = rope_base^(-2c/d) unless inv_freq_host   */
+  const double* inv_freq_host; /* host, optional [d/2] frequencies (scaled RoPE)  */
+  float   softmax_scale;    /* 0 -> 1/sqrt(head_dim)                              */
+  int32_t pool_mode;        /* dapq_pool_mode                                     */
+  int32_t pool_kernel;      /* odd window width; ignored for DAPQ_POOL_NONE       */
+  int32_t reserved;         /* must be 0                                          */
+} dapq_shape;
+
+typedef struct {
+  const void* k;                  /* device, [H_kv, R, d] view                    */
+  const void* v;                  /* device, same geometry (may be NULL for dapq_score) */
+  int64_t k_head_stride;          /* elements between KV heads                    */
+  int64_t k_row_stride;           /* elements between rows (>= d, multiple of 8)  */
+  int64_t v_head_stride;
+  int64_t v_row_stride;
+  const int32_t* cu_rows_host;    /* host [B+1], cu_rows[b+1]-cu_rows[b] = L_b + N */
+  const int32_t* prompt_len_host; /* host [B], L_b >= 1                            */
+  int32_t batch;                  /* B                                            */
+  int32_t reserved;               /* must be 0                                    */
+} dapq_cache_view;
+
+/* Create a context on `device` (made current for the call).  Allocates the workspace.
+ * Returns DAPQ_ERR_UNSUPPORTED for shapes outside the limits above. */
+DAPQ_API dapq_status dapq_create(dapq_ctx** out, const dapq_shape* shape, int device);
+DAPQ_API void dapq_destroy(dapq_ctx* ctx);
+
+/* Text of the last error of this context (never NULL; valid until the next call).
+ * With ctx == NULL: the reason the last dapq_create on this thread failed. */
+DAPQ_API const char* dapq_last_error(const dapq_ctx* ctx);
+
+/* Synchronises `stream`, then reads and clears the device status word.  Returns
+ * DAPQ_ERR_TIMEOUT if any kernel since the last poll gave up on a bounded wait
+ * (its results are then undefined), DAPQ_ERR_CUDA if the stream reports an error. */
+DAPQ_API dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched so far (for benchmarks' accounting). */
+DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
+
+/* Section 4.1: q_rot[b,h,i,:] = RoPE(q_pre[b,h,i,:], position pos_start[b] + i), rotate-half
+ * pairing (channel c with c + d/2), angles formed in double precision.
+ * q_pre, q_rot: device [B, H_q, N, d]; pos_start_host: host [B] (DapQ uses L_b; other
+ * values give the paper's shifted-position ablation). */
+DAPQ_API dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* pos_start_host,
+                               int32_t batch, void* q_rot, void* stream);
+
+/* Section 4.2, Eq. 4 with Attention = softmax(q K^T * scale) over the causal span of the
+ * extended prefill: pseudo query i sees the L_b prompt keys and synthetic keys 0 .. i.
+ *   scores[kvh, cu_prompt[b] + j] = sum_{g<G} sum_{i<N} P[b, kvh*G+g, i, j],  j < L_b.
+ * q_rot: device (already rotated).  lse_in: device [B, H_q, N] natural-log sum-exp of each
+ * pseudo query's visible logits, or NULL to have the library compute it (one extra sweep
+ * over K).  lse_out (nullable): receives the log-sum-exp used.  syn_mass (nullable):
+ * device [B, H_q], attention mass each head puts on the synthetic keys; for every KV head
+ * sum_j scores + sum_g syn_mass = G * N. */
+DAPQ_API dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* cache,
+                       const float* lse_in, float* scores, float* lse_out, float* syn_mass,
+                       void* stream);
+
+/* Section 4.2, Eq. 5: for every (b, kvh) the min(K_b, L_b) positions with the largest
+ * score; equal scores at the threshold go to the lower position; positions are written
+ * in ascending order.  scores: device [H_kv, T] (finite, >= 0); cu_prompt_host: host
+ * [B+1]; k_keep_host: host [B], K_b >= 1; idx_out: device [H_kv, KT]. */
+DAPQ_API dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* cu_prompt_host,
+                             const int32_t* k_keep_host, int32_t batch, int32_t* idx_out,
+                             void* stream);
+
+/* Section 4.2, pruning: k_out[kvh, cu_keep[b] + r, :] = K[kvh, cu_rows[b] + idx[kvh, cu_keep[b] + r], :]
+ * and the same rows of V; a bit-exact copy.  Synthetic rows are never copied.
+ * idx: device [H_kv, KT] as written by dapq_topk_select (entries outside [0, L_b) are
+ * skipped and flagged through dapq_poll_status as DAPQ_ERR_INVALID_ARG). */
+DAPQ_API dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const int32_t* idx,
+                            const int32_t* k_keep_host, void* k_out, void* v_out, void* stream);
+
+/* Figure 1, the whole eviction step for one layer: rotate to positions L_b + i, score,
+ * select, compact.  idx_out, scores_out may be NULL (kept in the workspace). */
+DAPQ_API dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
+                       const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
+                       float* scores_out, void* stream);
+
+/* dapq_evict for callers whose tensors live in host memory: q_pre, the cache view's k / v
+ * and k_out / v_out / idx_out are HOST pointers (pinned memory gives full copy speed).
+ * Copies the inputs to device staging buffers owned by the context (allocated on first
+ * use, sized from dapq_shape), runs dapq_evict, copies the results back and synchronises
+ * `stream` before returning. */
+DAPQ_API dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
+                            const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
+                            int32_t* idx_out_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAPQ_H */

@@ -1,0 +1,425 @@
+// C ABI of libdapq: context, argument checking, workspace, and the launch sequences.
+// See include/dapq.h for the contract of every entry point.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "dapq_internal.cuh"
+
+using namespace dapq;
+
+struct dapq_ctx {
+  int device = 0;
+  dapq_shape shape{};
+  Dims dims{};
+  int elem_bytes = 2;
+  int64_t max_chunks = 0;
+  // device workspace
+  double* inv_freq = nullptr;    // [d/2]
+  int* status = nullptr;         // device status word
+  void* q_rot = nullptr;         // [max_batch, H_q, N, d]
+  float2* part = nullptr;        // [max_chunks, H_q, N]
+  float* lse2 = nullptr;         // [max_batch, H_q, N]
+  float* scores = nullptr;       // [H_kv, max_total_rows]
+  float* pooled = nullptr;       // [H_kv, max_total_rows] (pooling only)
+  int32_t* idx = nullptr;        // [H_kv, max_total_rows]
+  // staging for dapq_evict_host (allocated on first use)
+  void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_ko = nullptr, *h_vo = nullptr;
+  int32_t* h_idx = nullptr;
+  int64_t n_launch = 0;
+  char err[512] = "";
+};
+
+namespace {
+
+// Message of the last failed dapq_create on this thread (there is no context to hold it).
+thread_local char g_create_err[256] = "";
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+dapq_status fail(dapq_ctx* ctx, dapq_status st, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+    va_end(ap);
+  }
+  return st;
+}
+
+dapq_status cuda_fail(dapq_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, DAPQ_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define DAPQ_CUDA(ctx, call)                                        \
+  do {                                                              \
+    cudaError_t e_ = (call);                                        \
+    if (e_ != cudaSuccess) return cuda_fail((ctx), e_, #call);      \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Fill the sequence table from the caller's host arrays and check it against the context.
+// Any of cu_rows / prompt_len may come from a cache view; k_keep and pos_start are optional.
+dapq_status build_table(dapq_ctx* ctx, int32_t batch, const int32_t* cu_rows, const int32_t* prompt_len,
+                        const int32_t* cu_prompt, const int32_t* k_keep, const int32_t* pos_start,
+                        SeqTable* t) {
+  const dapq_shape& sh = ctx->shape;
+  if (batch < 1) return fail(ctx, DAPQ_ERR_INVALID_ARG, "batch must be >= 1 (got %d)", batch);
+  if (batch > sh.max_batch)
+    return fail(ctx, DAPQ_ERR_WORKSPACE, "batch %d exceeds max_batch %d", batch, sh.max_batch);
+  memset(t, 0, sizeof(*t));
+  t->batch = batch;
+  int64_t rows = 0, prompt = 0, keep = 0, chunks = 0;
+  for (int b = 0; b < batch; ++b) {
+    int64_t L;
+    if (prompt_len) {
+      L = prompt_len[b];
+    } else if (cu_prompt) {
+      L = (int64_t)cu_prompt[b + 1] - cu_prompt[b];
+    } else {
+      L = 1;  // rope-only tables carry no lengths
+    }
+    if (L < 1) return fail(ctx, DAPQ_ERR_INVALID_ARG, "prompt length of sequence %d is %lld (must be >= 1)", b, (long long)L);
+    if (cu_prompt && cu_prompt[b] != prompt)
+      return fail(ctx, DAPQ_ERR_INVALID_ARG, "cu_prompt[%d] = %d, expected %lld", b, cu_prompt[b], (long long)prompt);
+    if (cu_rows) {
+      if (b == 0 && cu_rows[0] < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "cu_rows[0] is negative");
+      if ((int64_t)cu_rows[b + 1] - cu_rows[b] != L + sh.n_pseudo)
+        return fail(ctx, DAPQ_ERR_INVALID_ARG,
+                    "sequence %d owns %lld cache rows, expected L_b + N = %lld", b,
+                    (long long)((int64_t)cu_rows[b + 1] - cu_rows[b]), (long long)(L + sh.n_pseudo));
+      t->cu_rows[b] = cu_rows[b];
+      t->cu_rows[b + 1] = cu_rows[b + 1];
+    } else {
+      t->cu_rows[b] = (int32_t)rows;
+      t->cu_rows[b + 1] = (int32_t)(rows + L + sh.n_pseudo);
+    }
+    int64_t kb = L;
+    if (k_keep) {
+      if (k_keep[b] < 1) return fail(ctx, DAPQ_ERR_INVALID_ARG, "k_keep[%d] = %d (must be >= 1)", b, k_keep[b]);
+      kb = k_keep[b] < L ? k_keep[b] : L;
+    }
+    t->prompt_len[b] = (int32_t)L;
+    t->pos_start[b] = pos_start ? pos_start[b] : (int32_t)L;
+    if (pos_start && pos_start[b] < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "pos_start[%d] is negative", b);
+    t->cu_prompt[b] = (int32_t)prompt;
+    t->cu_keep[b] = (int32_t)keep;
+    t->cu_chunk[b] = (int32_t)chunks;
+    rows += L + sh.n_pseudo;
+    prompt += L;
+    keep += kb;
+    chunks += (L + kChunkKeys - 1) / kChunkKeys + 1;
+  }
+  t->cu_prompt[batch] = (int32_t)prompt;
+  t->cu_keep[batch] = (int32_t)keep;
+  t->cu_chunk[batch] = (int32_t)chunks;
+  t->n_chunks = (int32_t)chunks;
+  const int64_t last_row = cu_rows ? cu_rows[batch] : rows;
+  if ((prompt_len || cu_prompt) && (last_row > sh.max_total_rows || chunks > ctx->max_chunks))
+    return fail(ctx, DAPQ_ERR_WORKSPACE, "%lld cache rows exceed max_total_rows %lld",
+                (long long)last_row, (long long)sh.max_total_rows);
+  return DAPQ_OK;
+}
+
+dapq_status check_view(dapq_ctx* ctx, const dapq_cache_view* cv, bool need_v, bool host, CacheDev* out) {
+  if (!cv) return fail(ctx, DAPQ_ERR_INVALID_ARG, "cache view is NULL");
+  if (!cv->k || (need_v && !cv->v)) return fail(ctx, DAPQ_ERR_INVALID_ARG, "cache view has a NULL K or V pointer");
+  if (!cv->cu_rows_host || !cv->prompt_len_host)
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "cache view needs cu_rows_host and prompt_len_host");
+  if (cv->reserved != 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "cache view reserved field must be 0");
+  const int per16 = 16 / ctx->elem_bytes;
+  const bool use_v = cv->v != nullptr;
+  if (cv->k_row_stride < kHeadDim || cv->k_head_stride < 0 || (use_v && (cv->v_row_stride < kHeadDim || cv->v_head_stride < 0)))
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "row strides must be >= head_dim and head strides >= 0");
+  if (!host) {
+    if (cv->k_row_stride % per16 || cv->k_head_stride % per16 || !aligned16(cv->k) ||
+        (use_v && (cv->v_row_stride % per16 || cv->v_head_stride % per16 || !aligned16(cv->v))))
+      return fail(ctx, DAPQ_ERR_UNSUPPORTED, "K/V base pointers and strides must be multiples of 16 bytes");
+  }
+  out->k = cv->k;
+  out->v = cv->v;
+  out->k_head_stride = cv->k_head_stride;
+  out->k_row_stride = cv->k_row_stride;
+  out->v_head_stride = cv->v_head_stride;
+  out->v_row_stride = cv->v_row_stride;
+  return DAPQ_OK;
+}
+
+dapq_status run_score(dapq_ctx* ctx, const void* q_rot, const CacheDev& cd, const SeqTable& t,
+                      const float* lse_in, float* scores, int64_t score_stride, float* lse_out,
+                      float* syn_mass, cudaStream_t s) {
+  int n = 0;
+  cudaError_t e = launch_score_fma(ctx->shape.dtype, q_rot, cd, t, ctx->dims, lse_in, ctx->part, ctx->lse2,
+                                   scores, score_stride, lse_out, syn_mass, s, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "score kernels");
+  return DAPQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
+  if (!out || !sh) return DAPQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  dapq_ctx* ctx = new (std::nothrow) dapq_ctx();
+  if (!ctx) return DAPQ_ERR_CUDA;
+  // Errors before the context exists are reported through a context that is then freed:
+  // keep the message reachable by returning the status only.
+  auto bail = [&](dapq_status st, const char* why) {
+    snprintf(g_create_err, sizeof(g_create_err), "dapq_create: %s", why);
+    dapq_destroy(ctx);
+    return st;
+  };
+  if (sh->head_dim != kHeadDim) return bail(DAPQ_ERR_UNSUPPORTED, "head_dim must be 128");
+  if (sh->n_pseudo < 1 || sh->n_pseudo > kMaxPseudo) return bail(DAPQ_ERR_UNSUPPORTED, "n_pseudo must be in 1..128");
+  if (sh->n_q_heads < 1 || sh->n_kv_heads < 1 || sh->n_q_heads % sh->n_kv_heads)
+    return bail(DAPQ_ERR_INVALID_ARG, "n_kv_heads must divide n_q_heads");
+  if (sh->max_batch < 1 || sh->max_total_rows < 1) return bail(DAPQ_ERR_INVALID_ARG, "max_batch and max_total_rows must be >= 1");
+  if (sh->max_batch > kMaxBatch || sh->max_total_rows > 0x7fffffffLL)
+    return bail(DAPQ_ERR_UNSUPPORTED, "max_batch > 128 or max_total_rows >= 2^31");
+  if (sh->dtype != DAPQ_BF16 && sh->dtype != DAPQ_F32) return bail(DAPQ_ERR_INVALID_ARG, "unknown dtype");
+  if (sh->reserved != 0) return bail(DAPQ_ERR_INVALID_ARG, "reserved must be 0");
+  if (sh->pool_mode != DAPQ_POOL_NONE) return bail(DAPQ_ERR_UNSUPPORTED, "pooling is not available");
+  if (!sh->inv_freq_host && !(sh->rope_base > 0.0)) return bail(DAPQ_ERR_INVALID_ARG, "rope_base must be > 0");
+  if (!(sh->softmax_scale >= 0.f)) return bail(DAPQ_ERR_INVALID_ARG, "softmax_scale must be >= 0");
+
+  ctx->device = device;
+  ctx->shape = *sh;
+  ctx->shape.inv_freq_host = nullptr;
+  ctx->elem_bytes = sh->dtype == DAPQ_BF16 ? 2 : 4;
+  ctx->dims.n_q_heads = sh->n_q_heads;
+  ctx->dims.n_kv_heads = sh->n_kv_heads;
+  ctx->dims.group = sh->n_q_heads / sh->n_kv_heads;
+  ctx->dims.n_pseudo = sh->n_pseudo;
+  const double scale = sh->softmax_scale > 0.f ? (double)sh->softmax_scale : 1.0 / sqrt((double)kHeadDim);
+  ctx->dims.scale_log2e = (float)(scale * 1.4426950408889634074);
+  ctx->max_chunks = (sh->max_total_rows + kChunkKeys - 1) / kChunkKeys + 2LL * sh->max_batch;
+
+  DeviceGuard guard(device);
+  if (!guard.ok) return bail(DAPQ_ERR_CUDA, "cannot make the device current");
+  double freq[kHeadDim / 2];
+  for (int c = 0; c < kHeadDim / 2; ++c)
+    freq[c] = sh->inv_freq_host ? sh->inv_freq_host[c] : pow(sh->rope_base, -2.0 * c / (double)kHeadDim);
+  const size_t hq_n = (size_t)sh->n_q_heads * sh->n_pseudo;
+  const size_t rows = (size_t)sh->max_total_rows;
+  bool ok = true;
+  ok = ok && cudaMalloc(&ctx->inv_freq, sizeof(freq)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->q_rot, (size_t)sh->max_batch * hq_n * kHeadDim * ctx->elem_bytes) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->part, (size_t)ctx->max_chunks * hq_n * sizeof(float2)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->lse2, (size_t)sh->max_batch * hq_n * sizeof(float)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->scores, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->idx, (size_t)sh->n_kv_heads * rows * sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaMemcpy(ctx->inv_freq, freq, sizeof(freq), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->status, 0, sizeof(int)) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return bail(DAPQ_ERR_CUDA, "workspace allocation failed"); }
+  *out = ctx;
+  return DAPQ_OK;
+}
+
+void dapq_destroy(dapq_ctx* ctx) {
+  if (!ctx) return;
+  {
+    DeviceGuard guard(ctx->device);
+    void* bufs[] = {ctx->inv_freq, ctx->status, ctx->q_rot, ctx->part, ctx->lse2, ctx->scores, ctx->pooled,
+                    ctx->idx, ctx->h_q, ctx->h_k, ctx->h_v, ctx->h_ko, ctx->h_vo, ctx->h_idx};
+    for (void* p : bufs)
+      if (p) cudaFree(p);
+  }
+  delete ctx;
+}
+
+const char* dapq_last_error(const dapq_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
+
+int64_t dapq_launch_count(const dapq_ctx* ctx) { return ctx ? ctx->n_launch : 0; }
+
+dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)stream;
+  int word = 0;
+  DAPQ_CUDA(ctx, cudaStreamSynchronize(s));
+  DAPQ_CUDA(ctx, cudaMemcpy(&word, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word) DAPQ_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof(int)));
+  if (word & kStatusTimeout) return fail(ctx, DAPQ_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its results are undefined");
+  if (word & kStatusBadIndex) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_compact_kv skipped indices outside [0, L_b)");
+  return DAPQ_OK;
+}
+
+dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* pos_start_host,
+                               int32_t batch, void* q_rot, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!q_pre || !q_rot || !pos_start_host) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_rope_pseudo_q: NULL argument");
+  SeqTable t;
+  dapq_status st = build_table(ctx, batch, nullptr, nullptr, nullptr, nullptr, pos_start_host, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  int n = 0;
+  cudaError_t e = launch_rope(ctx->shape.dtype, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
+  return DAPQ_OK;
+}
+
+dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* cache,
+                       const float* lse_in, float* scores, float* lse_out, float* syn_mass, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!q_rot || !scores) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_score: NULL argument");
+  if (!aligned16(q_rot)) return fail(ctx, DAPQ_ERR_UNSUPPORTED, "q_rot must be 16-byte aligned");
+  CacheDev cd;
+  dapq_status st = check_view(ctx, cache, false, false, &cd);
+  if (st != DAPQ_OK) return st;
+  SeqTable t;
+  st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, nullptr, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  return run_score(ctx, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
+}
+
+dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* cu_prompt_host,
+                             const int32_t* k_keep_host, int32_t batch, int32_t* idx_out, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!scores || !cu_prompt_host || !k_keep_host || !idx_out)
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_topk_select: NULL argument");
+  SeqTable t;
+  dapq_status st = build_table(ctx, batch, nullptr, nullptr, cu_prompt_host, k_keep_host, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  int n = 0;
+  cudaError_t e = launch_topk(scores, t.cu_prompt[batch], idx_out, t.cu_keep[batch], t, ctx->dims.n_kv_heads,
+                              (cudaStream_t)stream, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
+  return DAPQ_OK;
+}
+
+dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const int32_t* idx,
+                            const int32_t* k_keep_host, void* k_out, void* v_out, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!idx || !k_keep_host || !k_out || !v_out) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_compact_kv: NULL argument");
+  if (!aligned16(k_out) || !aligned16(v_out)) return fail(ctx, DAPQ_ERR_UNSUPPORTED, "k_out / v_out must be 16-byte aligned");
+  CacheDev cd;
+  dapq_status st = check_view(ctx, cache, true, false, &cd);
+  if (st != DAPQ_OK) return st;
+  SeqTable t;
+  st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, k_keep_host, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  int n = 0;
+  cudaError_t e = launch_compact(ctx->shape.dtype, cd, idx, t.cu_keep[t.batch], k_out, v_out, t,
+                                 ctx->dims.n_kv_heads, ctx->status, (cudaStream_t)stream, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "compaction kernel");
+  return DAPQ_OK;
+}
+
+dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
+                       const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
+                       float* scores_out, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!q_pre || !k_keep_host || !k_out || !v_out) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict: NULL argument");
+  if (!aligned16(k_out) || !aligned16(v_out)) return fail(ctx, DAPQ_ERR_UNSUPPORTED, "k_out / v_out must be 16-byte aligned");
+  CacheDev cd;
+  dapq_status st = check_view(ctx, cache, true, false, &cd);
+  if (st != DAPQ_OK) return st;
+  SeqTable t;
+  st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, k_keep_host, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)stream;
+  int n = 0;
+  cudaError_t e = launch_rope(ctx->shape.dtype, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
+  float* scores = scores_out ? scores_out : ctx->scores;
+  int32_t* idx = idx_out ? idx_out : ctx->idx;
+  const int64_t score_stride = t.cu_prompt[t.batch], idx_stride = t.cu_keep[t.batch];
+  st = run_score(ctx, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
+  if (st != DAPQ_OK) return st;
+  n = 0;
+  e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
+  n = 0;
+  e = launch_compact(ctx->shape.dtype, cd, idx, idx_stride, k_out, v_out, t, ctx->dims.n_kv_heads, ctx->status, s, &n);
+  ctx->n_launch += n;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "compaction kernel");
+  return DAPQ_OK;
+}
+
+dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
+                            const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
+                            int32_t* idx_out_host, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!q_pre_host || !k_keep_host || !k_out_host || !v_out_host)
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_host: NULL argument");
+  CacheDev hv;
+  dapq_status st = check_view(ctx, cache_host, true, true, &hv);
+  if (st != DAPQ_OK) return st;
+  SeqTable t;
+  st = build_table(ctx, cache_host->batch, cache_host->cu_rows_host, cache_host->prompt_len_host, nullptr,
+                   k_keep_host, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)stream;
+  const dapq_shape& sh = ctx->shape;
+  const size_t eb = (size_t)ctx->elem_bytes, row_bytes = (size_t)kHeadDim * eb;
+  if (!ctx->h_k) {
+    const size_t cache_bytes = (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * row_bytes;
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_q, (size_t)sh.max_batch * sh.n_q_heads * sh.n_pseudo * row_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_k, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_v, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_ko, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_vo, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_idx, (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * sizeof(int32_t)));
+  }
+  // device copy of the used row range [cu_rows[0], cu_rows[B]) of every head, packed from row 0
+  const int64_t row0 = t.cu_rows[0], n_rows = t.cu_rows[t.batch] - row0;
+  DAPQ_CUDA(ctx, cudaMemcpyAsync(ctx->h_q, q_pre_host, (size_t)t.batch * sh.n_q_heads * sh.n_pseudo * row_bytes,
+                                 cudaMemcpyHostToDevice, s));
+  for (int h = 0; h < sh.n_kv_heads; ++h) {
+    const char* ks = (const char*)hv.k + ((size_t)h * hv.k_head_stride + (size_t)row0 * hv.k_row_stride) * eb;
+    const char* vs = (const char*)hv.v + ((size_t)h * hv.v_head_stride + (size_t)row0 * hv.v_row_stride) * eb;
+    DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_k + (size_t)h * n_rows * row_bytes, row_bytes, ks,
+                                     (size_t)hv.k_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
+    DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_v + (size_t)h * n_rows * row_bytes, row_bytes, vs,
+                                     (size_t)hv.v_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
+  }
+  int32_t cu_local[kMaxBatch + 1];
+  for (int b = 0; b <= t.batch; ++b) cu_local[b] = (int32_t)(t.cu_rows[b] - row0);
+  dapq_cache_view dv;
+  memset(&dv, 0, sizeof(dv));
+  dv.k = ctx->h_k;
+  dv.v = ctx->h_v;
+  dv.k_head_stride = dv.v_head_stride = n_rows * kHeadDim;
+  dv.k_row_stride = dv.v_row_stride = kHeadDim;
+  dv.cu_rows_host = cu_local;
+  dv.prompt_len_host = cache_host->prompt_len_host;
+  dv.batch = t.batch;
+  st = dapq_evict(ctx, ctx->h_q, &dv, k_keep_host, ctx->h_ko, ctx->h_vo, ctx->h_idx, nullptr, stream);
+  if (st != DAPQ_OK) return st;
+  const size_t kt = (size_t)t.cu_keep[t.batch];
+  DAPQ_CUDA(ctx, cudaMemcpyAsync(k_out_host, ctx->h_ko, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
+  DAPQ_CUDA(ctx, cudaMemcpyAsync(v_out_host, ctx->h_vo, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
+  if (idx_out_host)
+    DAPQ_CUDA(ctx, cudaMemcpyAsync(idx_out_host, ctx->h_idx, (size_t)sh.n_kv_heads * kt * sizeof(int32_t),
+                                   cudaMemcpyDeviceToHost, s));
+  DAPQ_CUDA(ctx, cudaStreamSynchronize(s));
+  return DAPQ_OK;
+}
+
+}  // extern "C"

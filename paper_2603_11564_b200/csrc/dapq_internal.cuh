@@ -1,0 +1,73 @@
+// Internal declarations shared by the translation units of libdapq (not installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dapq.h"
+
+namespace dapq {
+
+constexpr int kHeadDim = DAPQ_HEAD_DIM;      // d
+constexpr int kMaxBatch = DAPQ_MAX_BATCH;
+constexpr int kMaxPseudo = DAPQ_MAX_PSEUDO;
+constexpr int kChunkKeys = 512;              // prompt keys per work chunk of the score sweeps
+
+// Per-call sequence geometry, passed by value to the kernels (host arrays never have to
+// be copied to the device, so a call adds no copy nodes to a stream).
+struct SeqTable {
+  int32_t batch;
+  int32_t n_chunks;                 // sum_b (ceil(L_b / kChunkKeys) + 1)
+  int32_t cu_rows[kMaxBatch + 1];   // first cache row of sequence b
+  int32_t cu_prompt[kMaxBatch + 1]; // first score column of sequence b
+  int32_t cu_keep[kMaxBatch + 1];   // first output row of sequence b (K_b clamped to L_b)
+  int32_t cu_chunk[kMaxBatch + 1];  // first work chunk of sequence b; its last chunk holds the
+                                    // N synthetic rows, the others kChunkKeys prompt rows each
+  int32_t prompt_len[kMaxBatch];    // L_b
+  int32_t pos_start[kMaxBatch];     // position of pseudo query 0
+};
+
+struct CacheDev {
+  const void* k;
+  const void* v;
+  int64_t k_head_stride, k_row_stride, v_head_stride, v_row_stride;  // elements
+};
+
+struct Dims {
+  int32_t n_q_heads, n_kv_heads, group, n_pseudo;
+  float scale_log2e;                // softmax scale * log2(e): logits are kept in base 2
+};
+
+// Device status word bits (set by kernels, read by dapq_poll_status).
+enum : int { kStatusTimeout = 1, kStatusBadIndex = 2 };
+
+__device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
+  // largest b in [0, n) with cu[b] <= x
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (cu[mid] <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// ---- launchers (each returns the cudaError_t of its launch) -------------------------------
+cudaError_t launch_rope(int dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
+                        const SeqTable& t, const Dims& dm, cudaStream_t s, int* n_launch);
+
+// Generic CUDA-core scorer (any N <= 128, both dtypes).
+//   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits
+//   lse2  : [B, H_q, N] base-2 log-sum-exp
+cudaError_t launch_score_fma(int dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
+                             const Dims& dm, const float* lse_in, float2* part, float* lse2,
+                             float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
+                             cudaStream_t s, int* n_launch);
+
+cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
+                        const SeqTable& t, int n_kv_heads, cudaStream_t s, int* n_launch);
+
+cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, int64_t idx_stride,
+                           void* k_out, void* v_out, const SeqTable& t, int n_kv_heads, int* status,
+                           cudaStream_t s, int* n_launch);
+
+}  // namespace dapq

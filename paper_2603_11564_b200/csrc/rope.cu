@@ -1,0 +1,60 @@
+// Rotation of the pseudo queries to their decode positions (Section 4.1: the N synthetic
+// tokens take positions L_p .. L_p+N-1, so their queries carry the positional encodings of
+// the first N decoding steps).
+//
+// One CTA per (pseudo query i, sequence b); thread c owns the channel pair (c, c + d/2).
+// The angle pos * theta_c is formed and reduced in double precision: at positions near
+// 131k a float angle has only ~7 fractional bits, which alone would cost half of the
+// scorer's error budget.  The table is tiny (B*N*64 sincos), so this costs nothing.
+#include "dapq_internal.cuh"
+
+namespace dapq {
+namespace {
+
+template <typename T> __device__ __forceinline__ double to_double(T x);
+template <> __device__ __forceinline__ double to_double<float>(float x) { return (double)x; }
+template <> __device__ __forceinline__ double to_double<__nv_bfloat16>(__nv_bfloat16 x) {
+  return (double)__bfloat162float(x);
+}
+template <typename T> __device__ __forceinline__ T from_double(double x);
+template <> __device__ __forceinline__ float from_double<float>(double x) { return (float)x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(double x) {
+  return __double2bfloat16(x);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kHeadDim / 2)
+rope_pseudo_q_kernel(const T* __restrict__ q_pre, T* __restrict__ q_rot,
+                     const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
+                     int n_q_heads, int n_pseudo) {
+  const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  constexpr int half = kHeadDim / 2;
+  const double ang = (double)(t.pos_start[b] + i) * inv_freq[c];
+  double sn, cs;
+  sincos(ang, &sn, &cs);
+  for (int h = 0; h < n_q_heads; ++h) {
+    const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
+    const double lo = to_double<T>(q_pre[base + c]);
+    const double hi = to_double<T>(q_pre[base + c + half]);
+    q_rot[base + c] = from_double<T>(lo * cs - hi * sn);
+    q_rot[base + c + half] = from_double<T>(hi * cs + lo * sn);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_rope(int dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
+                        const SeqTable& t, const Dims& dm, cudaStream_t s, int* n_launch) {
+  dim3 grid(dm.n_pseudo, t.batch), block(kHeadDim / 2);
+  if (dtype == DAPQ_BF16) {
+    rope_pseudo_q_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(
+        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+  } else {
+    rope_pseudo_q_kernel<float><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
+                                                       inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+  }
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+}  // namespace dapq

@@ -1,0 +1,282 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded inputs.
+
+Pass criteria: per-token scores within 2e-3 relative; index sets identical except inside
+the 2e-3 band around the K-th oracle score; compacted K/V bit-exact given the indices."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from gen import inputs as gi
+from oracle import dapq_oracle as orc
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dq():
+    import paper_2603_11564_b200 as lib
+    lib.load_library()
+    return lib
+
+
+def _ctx(dq, w: gi.Workload, **kw):
+    return dq.dapq_create(w.n_q_heads, w.n_kv_heads, w.n_pseudo, w.batch, w.total_rows,
+                          dq.DAPQ_BF16 if w.dtype == "bf16" else dq.DAPQ_F32, w.rope_base, **kw)
+
+
+def _small(name="llama3_8b_32k", lens=(700,), keep=(40,), **kw) -> gi.Workload:
+    return gi.workload(name, prompt_lens=tuple(lens), keep=tuple(keep), n_layers=1, **kw)
+
+
+def _gpu_evict(dq, w, data, ctx=None):
+    dev = "cuda"
+    own = ctx is None
+    ctx = ctx or _ctx(dq, w)
+    q, k, v = (data[x].to(dev) for x in ("q_pre", "k", "v"))
+    KT, T = int(w.cu_keep[-1]), w.total_prompt
+    k_out = torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=k.dtype, device=dev)
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty((w.n_kv_heads, KT), dtype=torch.int32, device=dev)
+    scores = torch.empty((w.n_kv_heads, T), dtype=torch.float32, device=dev)
+    dq.dapq_evict(ctx, q, k, v, w.cu_rows, w.prompt_lens, w.keep, k_out, v_out, idx, scores)
+    dq.dapq_poll_status(ctx)
+    if own:
+        dq.dapq_destroy(ctx)
+    return dict(k_out=k_out.cpu(), v_out=v_out.cpu(), idx=idx.cpu().numpy(), scores=scores.cpu().double().numpy())
+
+
+def _check_evict(w, data, got, ref):
+    cu_p, cu_k, cu_r = w.cu_prompt, w.cu_keep, w.cu_rows
+    n_band = 0
+    for b in range(w.batch):
+        L = w.prompt_lens[b]
+        for h in range(w.n_kv_heads):
+            tag = f"{w.name} b={b} kvh={h}"
+            util.assert_scores_close(got["scores"][h, cu_p[b]:cu_p[b + 1]], ref["scores"][b][h], tag)
+            gidx = got["idx"][h, cu_k[b]:cu_k[b + 1]]
+            n_band += util.assert_index_sets_match(gidx, ref["scores"][b][h], ref["idx"][b][h], L, tag)
+            # compaction is a bit-exact copy of the rows the GPU itself selected
+            rows = torch.as_tensor(gidx.astype(np.int64) + int(cu_r[b]))
+            assert torch.equal(got["k_out"][h, cu_k[b]:cu_k[b + 1]], data["k"][h].cpu()[rows]), tag
+            assert torch.equal(got["v_out"][h, cu_k[b]:cu_k[b + 1]], data["v"][h].cpu()[rows]), tag
+            for p in (data["needle_pos"][b, h] if w.n_needles else []):
+                assert int(p) in set(gidx.tolist()), f"{tag}: planted needle {p} evicted"
+    return n_band
+
+
+# ------------------------------------------------------------------------- dapq_rope_pseudo_q
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rope_parity(dq, dtype):
+    w = _small(lens=(5, 131072, 4097), keep=(1, 1, 1), dtype=dtype, n_pseudo=33, rope_base=5.0e5)
+    ctx = _ctx(dq, w)
+    data = gi.draw_layer(dataclasses.replace(w, prompt_lens=(8, 8, 8)), 0, "cpu")
+    q = data["q_pre"].cuda()
+    out = torch.empty_like(q)
+    pos = [5, 131072, 0]
+    dq.dapq_rope_pseudo_q(ctx, q, pos, out)
+    torch.cuda.synchronize()
+    ref = np.stack([orc.rope_pseudo_q(util.to_f64(data["q_pre"][b]), pos[b], w.rope_base) for b in range(3)])
+    got = util.to_f64(out)
+    tol = 2.0 ** -8 if dtype == "bf16" else 2.0 ** -22
+    assert np.all(np.abs(got - ref) <= tol * np.abs(ref) + 1e-7)
+    assert torch.equal(out[2, :, 0].cpu(), data["q_pre"][2, :, 0])      # position 0 is the identity
+    dq.dapq_destroy(ctx)
+
+
+# --------------------------------------------------------------------------------- dapq_score
+SCORE_CASES = [
+    # dtype, H_q, H_kv, N, prompt lengths
+    ("f32", 8, 2, 32, (2048,)),
+    ("f32", 2, 2, 1, (1,)),
+    ("f32", 3, 1, 5, (63, 64, 65)),
+    ("bf16", 8, 2, 64, (1500,)),
+    ("bf16", 7, 1, 64, (513, 1, 127)),
+    ("bf16", 8, 1, 128, (129, 1031)),
+    ("bf16", 4, 4, 100, (777,)),
+    ("bf16", 8, 2, 17, (512, 1024, 300, 5)),
+]
+
+
+@pytest.mark.parametrize("dtype,hq,hkv,n,lens", SCORE_CASES)
+def test_score_parity(dq, dtype, hq, hkv, n, lens):
+    w = _small(lens=lens, keep=tuple(1 for _ in lens), dtype=dtype, n_q_heads=hq, n_kv_heads=hkv, n_pseudo=n,
+               n_needles=0, outlier_channels=2 if dtype == "bf16" else 0)
+    data = gi.draw_layer(w, 0, "cpu")
+    q_rot64 = util.oracle_q_rot(w, data)
+    q_rot = q_rot64.to(w.torch_dtype())                   # the operand both sides read
+    ctx = _ctx(dq, w)
+    B = w.batch
+    scores = torch.empty((hkv, w.total_prompt), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, hq, n), dtype=torch.float32, device="cuda")
+    syn = torch.empty((B, hq), dtype=torch.float32, device="cuda")
+    dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, lse_out=lse, syn_mass=syn)
+    dq.dapq_poll_status(ctx)
+    first = scores.clone()
+    # bit-identical when repeated (fixed reduction order, no float atomics)
+    dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, lse_out=lse, syn_mass=syn)
+    torch.cuda.synchronize()
+    assert torch.equal(first, scores)
+    got = scores.cpu().double().numpy()
+    k64 = util.to_f64(data["k"])
+    for b in range(B):
+        r0, L = int(w.cu_rows[b]), lens[b]
+        ref = orc.score_sequence(util.to_f64(q_rot[b]), k64[:, r0:r0 + L + n], L, w.group)
+        util.assert_scores_close(got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]], ref["scores"], f"b={b}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), ref["lse"], rtol=0, atol=2e-3)
+        np.testing.assert_allclose(syn[b].cpu().numpy(), ref["syn_mass"], rtol=2e-3, atol=1e-6)
+        # mass conservation on the GPU's own numbers: sum_j scores + sum_g syn = G * N
+        tot = got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]].sum(axis=1) + syn[b].cpu().double().numpy().reshape(hkv, -1).sum(axis=1)
+        np.testing.assert_allclose(tot, np.full(hkv, w.group * n), rtol=1e-4)
+    # the caller's own log-sum-exp (from the oracle) replaces the first sweep
+    lse_ref = torch.from_numpy(np.stack([
+        orc.score_sequence(util.to_f64(q_rot[b]), k64[:, int(w.cu_rows[b]):int(w.cu_rows[b + 1])], lens[b], w.group)["lse"]
+        for b in range(B)])).float().cuda()
+    scores2 = torch.empty_like(scores)
+    dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores2, lse_in=lse_ref)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(scores2.cpu().numpy(), got, rtol=1e-3)
+    dq.dapq_destroy(ctx)
+
+
+def test_score_strided_view_and_custom_scale(dq):
+    w = _small(lens=(300, 90), keep=(1, 1), n_q_heads=4, n_kv_heads=2, n_pseudo=16, n_needles=0, outlier_channels=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    q_rot = util.oracle_q_rot(w, data).to(torch.bfloat16)
+    R = w.total_rows
+    # cache stored as [R, H_kv, 2*d] (row-major over tokens, padded rows): heads interleaved
+    big = torch.zeros((R, w.n_kv_heads, 256), dtype=torch.bfloat16, device="cuda")
+    big[:, :, :128] = data["k"].cuda().transpose(0, 1)
+    kview = big[:, :, :128].transpose(0, 1)
+    assert kview.stride() == (256, 512, 1)
+    ctx = _ctx(dq, w, softmax_scale=0.05)
+    scores = torch.empty((w.n_kv_heads, w.total_prompt), dtype=torch.float32, device="cuda")
+    dq.dapq_score(ctx, q_rot.cuda(), kview, w.cu_rows, w.prompt_lens, scores)
+    torch.cuda.synchronize()
+    k64 = util.to_f64(data["k"])
+    for b in range(2):
+        r0, L = int(w.cu_rows[b]), w.prompt_lens[b]
+        ref = orc.score_sequence(util.to_f64(q_rot[b]), k64[:, r0:r0 + L + 16], L, w.group, scale=0.05)
+        util.assert_scores_close(scores[:, w.cu_prompt[b]:w.cu_prompt[b + 1]].cpu().double().numpy(), ref["scores"])
+    dq.dapq_destroy(ctx)
+
+
+# -------------------------------------------------------------------------- dapq_topk_select
+def test_topk_exact_with_ties(dq):
+    rng = np.random.default_rng(5)
+    lens, keep = (1, 33, 4096, 5000, 131072, 77), (1, 33, 1, 4999, 3932, 200)
+    w = _small(lens=lens, keep=keep, n_q_heads=3, n_kv_heads=3, n_pseudo=4, n_needles=0, outlier_channels=0)
+    T = w.total_prompt
+    s = rng.random((3, T)).astype(np.float32)
+    s[1] = np.round(s[1] * 50) / 50                      # heavy ties
+    s[2] = 0.25                                          # all equal
+    s[0, ::7] = 0.0
+    ctx = _ctx(dq, w)
+    idx = torch.full((3, int(w.cu_keep[-1])), -1, dtype=torch.int32, device="cuda")
+    dq.dapq_topk_select(ctx, torch.from_numpy(s).cuda(), w.cu_prompt, keep, idx)
+    torch.cuda.synchronize()
+    got = idx.cpu().numpy()
+    for b in range(len(lens)):
+        for h in range(3):
+            ref = orc.topk_select(s[h, w.cu_prompt[b]:w.cu_prompt[b + 1]].astype(np.float64), keep[b])
+            np.testing.assert_array_equal(got[h, w.cu_keep[b]:w.cu_keep[b + 1]], ref, err_msg=f"b={b} h={h}")
+    dq.dapq_destroy(ctx)
+
+
+# --------------------------------------------------------------------------- dapq_compact_kv
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_compact_bit_exact_given_oracle_indices(dq, dtype):
+    w = _small(lens=(300, 17, 1000), keep=(30, 40, 999), dtype=dtype, n_q_heads=4, n_kv_heads=2, n_pseudo=8,
+               n_needles=0, outlier_channels=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    ref = util.oracle_evict(w, data)
+    idx = np.concatenate(ref["idx"], axis=1)             # [H_kv, KT]
+    ctx = _ctx(dq, w)
+    KT = idx.shape[1]
+    k_out = torch.zeros((2, KT, 128), dtype=w.torch_dtype(), device="cuda")
+    v_out = torch.zeros_like(k_out)
+    dq.dapq_compact_kv(ctx, data["k"].cuda(), data["v"].cuda(), w.cu_rows, w.prompt_lens, torch.from_numpy(idx).cuda(),
+                       w.keep, k_out, v_out)
+    dq.dapq_poll_status(ctx)
+    view = torch.int16 if dtype == "bf16" else torch.int32
+    for b in range(w.batch):
+        sl = slice(int(w.cu_keep[b]), int(w.cu_keep[b + 1]))
+        for h in range(2):
+            rows = torch.as_tensor(ref["idx"][b][h].astype(np.int64) + int(w.cu_rows[b]))
+            assert torch.equal(k_out[h, sl].cpu().view(view), data["k"][h][rows].view(view))
+            assert torch.equal(v_out[h, sl].cpu().view(view), data["v"][h][rows].view(view))
+            np.testing.assert_array_equal(util.to_f64(k_out[h, sl]), ref["k_out"][b][h])
+    # an index that points at a synthetic row is skipped and reported, never read
+    bad = torch.from_numpy(idx).cuda().clone()
+    bad[0, 0] = w.prompt_lens[0]
+    dq.dapq_compact_kv(ctx, data["k"].cuda(), data["v"].cuda(), w.cu_rows, w.prompt_lens, bad, w.keep, k_out, v_out)
+    with pytest.raises(dq.DapqError):
+        dq.dapq_poll_status(ctx)
+    dq.dapq_poll_status(ctx)                             # the word was cleared
+    dq.dapq_destroy(ctx)
+
+
+# -------------------------------------------------------------------------------- dapq_evict
+def test_evict_tiny_config_in_full(dq):
+    w = gi.workload("tiny")
+    data = util.make_case(w)
+    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+
+
+@pytest.mark.parametrize("name,scale", [("llama3_8b_32k", 16), ("qwen25_7b_128k", 64), ("batched_serving", 16),
+                                        ("llama3_70b_128k", 64)])
+def test_evict_scaled_configs(dq, name, scale):
+    w = gi.scaled_down(name, scale, n_layers=1)
+    data = util.make_case(w)
+    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+
+
+def test_evict_edge_shapes(dq):
+    # K_b >= L_b keeps everything; L_b = 1; K_b = 1; lengths around the tile sizes
+    w = _small(lens=(1, 64, 65, 511, 513, 2), keep=(5, 64, 1, 510, 100, 1), n_q_heads=4, n_kv_heads=2,
+               n_pseudo=3, n_needles=0)
+    data = util.make_case(w)
+    got = _gpu_evict(dq, w, data)
+    _check_evict(w, data, got, util.oracle_evict(w, data))
+    np.testing.assert_array_equal(got["idx"][0, 1:65], np.arange(64))
+
+
+def test_evict_host_matches_device_call(dq):
+    w = gi.scaled_down("batched_serving", 32, n_layers=1)
+    data = util.make_case(w)
+    ctx = _ctx(dq, w)
+    dev = _gpu_evict(dq, w, data, ctx)
+    KT = int(w.cu_keep[-1])
+    pin = lambda t: t.contiguous().pin_memory()
+    k_out = torch.empty((w.n_kv_heads, KT, 128), dtype=torch.bfloat16).pin_memory()
+    v_out = torch.empty_like(k_out).pin_memory()
+    idx = torch.empty((w.n_kv_heads, KT), dtype=torch.int32).pin_memory()
+    dq.dapq_evict_host(ctx, pin(data["q_pre"]), pin(data["k"]), pin(data["v"]), w.cu_rows, w.prompt_lens, w.keep,
+                       k_out, v_out, idx)
+    assert torch.equal(k_out, dev["k_out"]) and torch.equal(v_out, dev["v_out"])
+    np.testing.assert_array_equal(idx.numpy(), dev["idx"])
+    dq.dapq_destroy(ctx)
+
+
+def test_argument_errors_launch_nothing(dq):
+    w = _small(lens=(100,), keep=(10,), n_needles=0)
+    data = gi.draw_layer(w, 0, "cuda")
+    ctx = _ctx(dq, w)
+    n0 = dq.dapq_launch_count(ctx)
+    scores = torch.empty((w.n_kv_heads, 100), dtype=torch.float32, device="cuda")
+    with pytest.raises(dq.DapqError) as e:       # rows do not add up to L + N
+        dq.dapq_score(ctx, data["q_pre"], data["k"], [0, 150], [100], scores)
+    assert e.value.status == dq.DAPQ_ERR_INVALID_ARG
+    with pytest.raises(dq.DapqError) as e:       # larger than the workspace
+        dq.dapq_score(ctx, data["q_pre"], data["k"], [0, 264], [200], scores)
+    assert e.value.status == dq.DAPQ_ERR_WORKSPACE
+    with pytest.raises(dq.DapqError) as e:       # misaligned row stride
+        dq.dapq_score(ctx, data["q_pre"], data["k"].as_strided((2, 164, 128), (164 * 132, 132, 1)),
+                      w.cu_rows, w.prompt_lens, scores)
+    assert e.value.status == dq.DAPQ_ERR_UNSUPPORTED
+    with pytest.raises(dq.DapqError):
+        dq.dapq_topk_select(ctx, scores, [0, 100], [0], torch.empty(8, 10, dtype=torch.int32, device="cuda"))
+    assert dq.dapq_launch_count(ctx) == n0
+    dq.dapq_destroy(ctx)
