@@ -40,7 +40,7 @@ class Workload:
     rope_base: float
     seed: int
     n_needles: int = 0             # planted needle keys per KV head and sequence
-    needle_tau: float = 12.0       # mean logit of a needle against the window
+    needle_rho: float = 3.0        # norm of a needle key in units of sqrt(d) (a typical key has 1)
     outlier_channels: int = 0      # channels per KV head scaled by outlier_scale
     outlier_scale: float = 8.0
     sink_rows: int = 0             # first rows of each head with a heavy-tailed bias
@@ -182,10 +182,12 @@ def plant_structure(w: Workload, data: Dict[str, object], q_rot: torch.Tensor) -
 
     q_rot [B, H_q, N, d] are the pseudo queries ALREADY rotated to their decode
     positions, supplied by the caller.  With qbar the mean of the G*N rotated
-    queries of a KV head's group:
-      needle row:  k = alpha * qbar, alpha = tau*sqrt(d)/|qbar|^2, so that the mean
-                   logit of the window against the needle equals tau;
-      sink row j:  k += tau_j*sqrt(d)/|qbar| * qbar/|qbar|.
+    queries of a KV head's group and u = qbar/|qbar|:
+      needle row:  k = rho * sqrt(d) * u   (a scaled copy of the mean rotated query, rho = 3
+                   times the norm of a typical key, so every window query's logit against
+                   it is rho*(|qbar| + z), z ~ N(0,1): far above the bulk, yet a key norm
+                   a bf16 cache can hold without swamping the other rows' precision);
+      sink row j:  k += tau_j * u, tau_j = 6 + |t_2| clipped at 30 (heavy-tailed).
     Values are rounded to the storage dtype on assignment.
     """
     if not (w.n_needles or w.sink_rows):
@@ -197,14 +199,13 @@ def plant_structure(w: Workload, data: Dict[str, object], q_rot: torch.Tensor) -
     for b in range(w.batch):
         for h in range(w.n_kv_heads):
             qbar = q[b, h * G:(h + 1) * G].reshape(-1, d).mean(dim=0)
-            nrm2 = float((qbar * qbar).sum())
+            u = qbar / qbar.norm()
             if w.n_needles:
-                alpha = w.needle_tau * math.sqrt(d) / nrm2
                 rows = torch.as_tensor(data["needle_pos"][b, h] + int(cu[b]), device=k.device)
-                k[h, rows] = (alpha * qbar).to(k.dtype).unsqueeze(0).expand(len(rows), d)
+                k[h, rows] = (w.needle_rho * math.sqrt(d) * u).to(k.dtype).unsqueeze(0).expand(len(rows), d)
             for j in range(w.sink_rows):
                 tau = float(data["sink_tau"][b, h, j])
-                add = (tau * math.sqrt(d) / nrm2) * qbar
+                add = tau * u
                 row = int(cu[b]) + j
                 k[h, row] = (k[h, row].to(torch.float64) + add).to(k.dtype)
 

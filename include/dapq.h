@@ -122,6 +122,18 @@ DAPQ_API dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream);
 /* Number of kernels this context has launched so far (for benchmarks' accounting). */
 DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
 
+/* Per-kernel timing for benchmarks (the paper has no counterpart).  While enabled, every
+ * kernel launch is bracketed by CUDA events on its stream; dapq_profile(ctx, 1) also clears
+ * the totals.  dapq_profile_read synchronises `stream` and returns, per kernel kind, the
+ * summed device time in milliseconds and the number of launches since profiling was
+ * enabled.  ms_out / count_out: host [DAPQ_PROF_KINDS], in the order of dapq_prof_kind. */
+typedef enum {
+  DAPQ_PROF_ROPE = 0, DAPQ_PROF_SWEEP1 = 1, DAPQ_PROF_LSE_MERGE = 2, DAPQ_PROF_SWEEP2 = 3,
+  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_KINDS = 6
+} dapq_prof_kind;
+DAPQ_API dapq_status dapq_profile(dapq_ctx* ctx, int32_t enable);
+DAPQ_API dapq_status dapq_profile_read(dapq_ctx* ctx, void* stream, double* ms_out, int64_t* count_out);
+
 /* Section 4.1: q_rot[b,h,i,:] = RoPE(q_pre[b,h,i,:], position pos_start[b] + i), rotate-half
  * pairing (channel c with c + d/2), angles formed in double precision.
  * q_pre, q_rot: device [B, H_q, N, d]; pos_start_host: host [B] (DapQ uses L_b; other

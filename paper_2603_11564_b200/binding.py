@@ -25,7 +25,7 @@ _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORT
                  3: "DAPQ_ERR_WORKSPACE", 4: "DAPQ_ERR_CUDA", 5: "DAPQ_ERR_TIMEOUT"}
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
-           "dapq_launch_count", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
+           "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
            "dapq_compact_kv", "dapq_evict", "dapq_evict_host")
 
 
@@ -73,6 +73,10 @@ def load_library() -> C.CDLL:
     lib.dapq_poll_status.restype = C.c_int
     lib.dapq_launch_count.argtypes = [vp]
     lib.dapq_launch_count.restype = C.c_int64
+    lib.dapq_profile.argtypes = [vp, C.c_int32]
+    lib.dapq_profile.restype = C.c_int
+    lib.dapq_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.dapq_profile_read.restype = C.c_int
     lib.dapq_rope_pseudo_q.argtypes = [vp, vp, i32p, C.c_int32, vp, vp]
     lib.dapq_rope_pseudo_q.restype = C.c_int
     lib.dapq_score.argtypes = [vp, vp, C.POINTER(dapq_cache_view), f32p, f32p, f32p, f32p, vp]
@@ -160,6 +164,21 @@ def dapq_poll_status(ctx, stream=None) -> None:
 
 def dapq_launch_count(ctx) -> int:
     return int(load_library().dapq_launch_count(ctx))
+
+
+PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact")
+
+
+def dapq_profile(ctx, enable: bool) -> None:
+    _check(ctx, load_library().dapq_profile(ctx, 1 if enable else 0))
+
+
+def dapq_profile_read(ctx, stream=None):
+    """{kind: (total_ms, launches)} since profiling was enabled."""
+    ms = (C.c_double * len(PROF_KINDS))()
+    cnt = (C.c_int64 * len(PROF_KINDS))()
+    _check(ctx, load_library().dapq_profile_read(ctx, _stream(stream), ms, cnt))
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(PROF_KINDS)}
 
 
 def dapq_rope_pseudo_q(ctx, q_pre: torch.Tensor, pos_start: Sequence[int], q_rot: torch.Tensor,

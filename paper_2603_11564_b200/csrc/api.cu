@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "dapq_internal.cuh"
 
@@ -29,9 +30,40 @@ struct dapq_ctx {
   // staging for dapq_evict_host (allocated on first use)
   void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_ko = nullptr, *h_vo = nullptr;
   int32_t* h_idx = nullptr;
-  int64_t n_launch = 0;
+  LaunchLog log;
   char err[512] = "";
 };
+
+// ---- launch accounting and per-kernel event timing ----------------------------------------
+namespace dapq {
+struct ProfImpl {
+  std::vector<cudaEvent_t> pool;      // event pairs, reused after every drain
+  std::vector<int> kinds;             // kind of each pending pair
+  double ms[kKindCount] = {};
+  int64_t count[kKindCount] = {};
+  ~ProfImpl() { for (cudaEvent_t e : pool) cudaEventDestroy(e); }
+};
+
+void LaunchLog::begin(int kind, cudaStream_t s) {
+  ++n_launch;
+  if (!profiling) return;
+  ProfImpl* p = static_cast<ProfImpl*>(impl);
+  const size_t n = p->kinds.size();
+  while (p->pool.size() < 2 * (n + 1)) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) { profiling = false; return; }
+    p->pool.push_back(e);
+  }
+  p->kinds.push_back(kind);
+  cudaEventRecord(p->pool[2 * n], s);
+}
+
+void LaunchLog::end(cudaStream_t s) {
+  if (!profiling) return;
+  ProfImpl* p = static_cast<ProfImpl*>(impl);
+  cudaEventRecord(p->pool[2 * (p->kinds.size() - 1) + 1], s);
+}
+}  // namespace dapq
 
 namespace {
 
@@ -157,13 +189,11 @@ dapq_status check_view(dapq_ctx* ctx, const dapq_cache_view* cv, bool need_v, bo
   return DAPQ_OK;
 }
 
-dapq_status run_score(dapq_ctx* ctx, const void* q_rot, const CacheDev& cd, const SeqTable& t,
+dapq_status run_score(dapq_ctx* ctx, int q_dtype, const void* q_rot, const CacheDev& cd, const SeqTable& t,
                       const float* lse_in, float* scores, int64_t score_stride, float* lse_out,
                       float* syn_mass, cudaStream_t s) {
-  int n = 0;
-  cudaError_t e = launch_score_fma(ctx->shape.dtype, q_rot, cd, t, ctx->dims, lse_in, ctx->part, ctx->lse2,
-                                   scores, score_stride, lse_out, syn_mass, s, &n);
-  ctx->n_launch += n;
+  cudaError_t e = launch_score_fma(ctx->shape.dtype, q_dtype, q_rot, cd, t, ctx->dims, lse_in, ctx->part, ctx->lse2,
+                                   scores, score_stride, lse_out, syn_mass, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score kernels");
   return DAPQ_OK;
 }
@@ -219,7 +249,7 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   bool ok = true;
   ok = ok && cudaMalloc(&ctx->inv_freq, sizeof(freq)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->status, sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->q_rot, (size_t)sh->max_batch * hq_n * kHeadDim * ctx->elem_bytes) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->q_rot, (size_t)sh->max_batch * hq_n * kHeadDim * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->part, (size_t)ctx->max_chunks * hq_n * sizeof(float2)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->lse2, (size_t)sh->max_batch * hq_n * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->scores, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
@@ -240,12 +270,13 @@ void dapq_destroy(dapq_ctx* ctx) {
     for (void* p : bufs)
       if (p) cudaFree(p);
   }
+  delete static_cast<dapq::ProfImpl*>(ctx->log.impl);
   delete ctx;
 }
 
 const char* dapq_last_error(const dapq_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
 
-int64_t dapq_launch_count(const dapq_ctx* ctx) { return ctx ? ctx->n_launch : 0; }
+int64_t dapq_launch_count(const dapq_ctx* ctx) { return ctx ? ctx->log.n_launch : 0; }
 
 dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
@@ -260,6 +291,38 @@ dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream) {
   return DAPQ_OK;
 }
 
+dapq_status dapq_profile(dapq_ctx* ctx, int32_t enable) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!ctx->log.impl) {
+    ctx->log.impl = new (std::nothrow) dapq::ProfImpl();
+    if (!ctx->log.impl) return fail(ctx, DAPQ_ERR_CUDA, "out of host memory");
+  }
+  dapq::ProfImpl* p = static_cast<dapq::ProfImpl*>(ctx->log.impl);
+  if (enable) {
+    p->kinds.clear();
+    for (int k = 0; k < kKindCount; ++k) { p->ms[k] = 0.0; p->count[k] = 0; }
+  }
+  ctx->log.profiling = enable != 0;
+  return DAPQ_OK;
+}
+
+dapq_status dapq_profile_read(dapq_ctx* ctx, void* stream, double* ms_out, int64_t* count_out) {
+  if (!ctx || !ms_out || !count_out) return DAPQ_ERR_INVALID_ARG;
+  dapq::ProfImpl* p = static_cast<dapq::ProfImpl*>(ctx->log.impl);
+  if (!p) return fail(ctx, DAPQ_ERR_INVALID_ARG, "profiling was never enabled");
+  DeviceGuard guard(ctx->device);
+  DAPQ_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  for (size_t i = 0; i < p->kinds.size(); ++i) {
+    float ms = 0.f;
+    DAPQ_CUDA(ctx, cudaEventElapsedTime(&ms, p->pool[2 * i], p->pool[2 * i + 1]));
+    p->ms[p->kinds[i]] += ms;
+    p->count[p->kinds[i]] += 1;
+  }
+  p->kinds.clear();
+  for (int k = 0; k < kKindCount; ++k) { ms_out[k] = p->ms[k]; count_out[k] = p->count[k]; }
+  return DAPQ_OK;
+}
+
 dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* pos_start_host,
                                int32_t batch, void* q_rot, void* stream) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
@@ -268,9 +331,7 @@ dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* 
   dapq_status st = build_table(ctx, batch, nullptr, nullptr, nullptr, nullptr, pos_start_host, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  int n = 0;
-  cudaError_t e = launch_rope(ctx->shape.dtype, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &n);
-  ctx->n_launch += n;
+  cudaError_t e = launch_rope(ctx->shape.dtype, ctx->shape.dtype, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
   return DAPQ_OK;
 }
@@ -287,7 +348,7 @@ dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* 
   st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, nullptr, nullptr, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  return run_score(ctx, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
+  return run_score(ctx, ctx->shape.dtype, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
 }
 
 dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* cu_prompt_host,
@@ -299,10 +360,8 @@ dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* 
   dapq_status st = build_table(ctx, batch, nullptr, nullptr, cu_prompt_host, k_keep_host, nullptr, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  int n = 0;
   cudaError_t e = launch_topk(scores, t.cu_prompt[batch], idx_out, t.cu_keep[batch], t, ctx->dims.n_kv_heads,
-                              (cudaStream_t)stream, &n);
-  ctx->n_launch += n;
+                              (cudaStream_t)stream, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
   return DAPQ_OK;
 }
@@ -319,10 +378,8 @@ dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const i
   st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, k_keep_host, nullptr, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  int n = 0;
   cudaError_t e = launch_compact(ctx->shape.dtype, cd, idx, t.cu_keep[t.batch], k_out, v_out, t,
-                                 ctx->dims.n_kv_heads, ctx->status, (cudaStream_t)stream, &n);
-  ctx->n_launch += n;
+                                 ctx->dims.n_kv_heads, ctx->status, (cudaStream_t)stream, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "compaction kernel");
   return DAPQ_OK;
 }
@@ -341,22 +398,17 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)stream;
-  int n = 0;
-  cudaError_t e = launch_rope(ctx->shape.dtype, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &n);
-  ctx->n_launch += n;
+  // the CUDA-core scorer reads the rotated queries unrounded (fp32)
+  cudaError_t e = launch_rope(ctx->shape.dtype, DAPQ_F32, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
   float* scores = scores_out ? scores_out : ctx->scores;
   int32_t* idx = idx_out ? idx_out : ctx->idx;
   const int64_t score_stride = t.cu_prompt[t.batch], idx_stride = t.cu_keep[t.batch];
-  st = run_score(ctx, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
+  st = run_score(ctx, DAPQ_F32, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
   if (st != DAPQ_OK) return st;
-  n = 0;
-  e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &n);
-  ctx->n_launch += n;
+  e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
-  n = 0;
-  e = launch_compact(ctx->shape.dtype, cd, idx, idx_stride, k_out, v_out, t, ctx->dims.n_kv_heads, ctx->status, s, &n);
-  ctx->n_launch += n;
+  e = launch_compact(ctx->shape.dtype, cd, idx, idx_stride, k_out, v_out, t, ctx->dims.n_kv_heads, ctx->status, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "compaction kernel");
   return DAPQ_OK;
 }

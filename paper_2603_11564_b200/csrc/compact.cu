@@ -40,7 +40,8 @@ compact_kv_kernel(const CacheDev cv, int elem_bytes, const int32_t* __restrict__
 
 cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, int64_t idx_stride,
                            void* k_out, void* v_out, const SeqTable& t, int n_kv_heads, int* status,
-                           cudaStream_t s, int* n_launch) {
+                           cudaStream_t s, LaunchLog* log) {
+  log->begin(kKindCompact, s);
   const int kt = t.cu_keep[t.batch];
   if (dtype == DAPQ_BF16) {
     constexpr int P = kHeadDim * 2 / 16;
@@ -53,7 +54,7 @@ cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, in
     compact_kv_kernel<P><<<grid, kCompactThreads, 0, s>>>(cv, 4, idx, idx_stride, (uint4*)k_out,
                                                           (uint4*)v_out, t, status);
   }
-  ++*n_launch;
+  log->end(s);
   return cudaGetLastError();
 }
 

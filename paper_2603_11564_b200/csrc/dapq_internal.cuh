@@ -51,23 +51,39 @@ __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
   return lo;
 }
 
+// Kernel kinds, for launch accounting and the optional per-kernel event timing.
+enum KernelKind : int { kKindRope = 0, kKindSweep1, kKindLseMerge, kKindSweep2, kKindTopk, kKindCompact,
+                        kKindCount };
+
+// Counts launches and, while profiling is on, brackets every launch with CUDA events on
+// the launching stream (implemented in api.cu; events come from a host-side pool).
+struct LaunchLog {
+  int64_t n_launch = 0;
+  bool profiling = false;
+  void* impl = nullptr;
+  void begin(int kind, cudaStream_t s);
+  void end(cudaStream_t s);
+};
+
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------
-cudaError_t launch_rope(int dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
-                        const SeqTable& t, const Dims& dm, cudaStream_t s, int* n_launch);
+// q_pre has element type `dtype`; q_rot is written as `out_dtype` (fp32 keeps the rotated
+// queries unrounded for the CUDA-core scorer).
+cudaError_t launch_rope(int dtype, int out_dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
+                        const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log);
 
 // Generic CUDA-core scorer (any N <= 128, both dtypes).
 //   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits
 //   lse2  : [B, H_q, N] base-2 log-sum-exp
-cudaError_t launch_score_fma(int dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
+cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
                              const Dims& dm, const float* lse_in, float2* part, float* lse2,
                              float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
-                             cudaStream_t s, int* n_launch);
+                             cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
-                        const SeqTable& t, int n_kv_heads, cudaStream_t s, int* n_launch);
+                        const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, int64_t idx_stride,
                            void* k_out, void* v_out, const SeqTable& t, int n_kv_heads, int* status,
-                           cudaStream_t s, int* n_launch);
+                           cudaStream_t s, LaunchLog* log);
 
 }  // namespace dapq

@@ -22,9 +22,9 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(
   return __double2bfloat16(x);
 }
 
-template <typename T>
+template <typename T, typename TO>
 __global__ void __launch_bounds__(kHeadDim / 2)
-rope_pseudo_q_kernel(const T* __restrict__ q_pre, T* __restrict__ q_rot,
+rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
                      int n_q_heads, int n_pseudo) {
   const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
@@ -36,24 +36,28 @@ rope_pseudo_q_kernel(const T* __restrict__ q_pre, T* __restrict__ q_rot,
     const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
     const double lo = to_double<T>(q_pre[base + c]);
     const double hi = to_double<T>(q_pre[base + c + half]);
-    q_rot[base + c] = from_double<T>(lo * cs - hi * sn);
-    q_rot[base + c + half] = from_double<T>(hi * cs + lo * sn);
+    q_rot[base + c] = from_double<TO>(lo * cs - hi * sn);
+    q_rot[base + c + half] = from_double<TO>(hi * cs + lo * sn);
   }
 }
 
 }  // namespace
 
-cudaError_t launch_rope(int dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
-                        const SeqTable& t, const Dims& dm, cudaStream_t s, int* n_launch) {
+cudaError_t launch_rope(int dtype, int out_dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
+                        const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log) {
+  log->begin(kKindRope, s);
   dim3 grid(dm.n_pseudo, t.batch), block(kHeadDim / 2);
-  if (dtype == DAPQ_BF16) {
-    rope_pseudo_q_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(
+  if (dtype == DAPQ_BF16 && out_dtype == DAPQ_BF16) {
+    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, block, 0, s>>>(
         (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+  } else if (dtype == DAPQ_BF16) {
+    rope_pseudo_q_kernel<__nv_bfloat16, float><<<grid, block, 0, s>>>(
+        (const __nv_bfloat16*)q_pre, (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
   } else {
-    rope_pseudo_q_kernel<float><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
-                                                       inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+    rope_pseudo_q_kernel<float, float><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
+                                                              inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
   }
-  ++*n_launch;
+  log->end(s);
   return cudaGetLastError();
 }
 

@@ -73,9 +73,9 @@ constexpr size_t fma_smem_bytes() {
 
 // grid (n_chunks, H_kv).  Thread (ty, tx) owns query rows ty + 16 r (r < R) and the keys
 // kk * 16 + tx (kk < 4) of each 64-key tile.
-template <typename T, int R, bool kSweep2>
+template <typename TQ, typename T, int R, bool kSweep2>
 __global__ void __launch_bounds__(kThreads)
-score_fma_kernel(const T* __restrict__ q_rot, const CacheDev cv, const __grid_constant__ SeqTable t,
+score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_constant__ SeqTable t,
                  const Dims dm, float2* __restrict__ part, const float* __restrict__ lse2,
                  float* __restrict__ scores, int64_t score_stride, float* __restrict__ syn_mass) {
   extern __shared__ __align__(16) float smem[];
@@ -105,7 +105,7 @@ score_fma_kernel(const T* __restrict__ q_rot, const CacheDev cv, const __grid_co
   for (int g = 0; g < G; ++g) {
     const int h = kvh * G + g;
     __syncthreads();                                        // Qs, lse_s, colacc free
-    stage_rows<T>(Qs, q_rot + ((int64_t)b * Hq + h) * N * kHeadDim, kHeadDim, N, 16 * R);
+    stage_rows<TQ>(Qs, q_rot + ((int64_t)b * Hq + h) * N * kHeadDim, kHeadDim, N, 16 * R);
     if (kSweep2) {
       for (int x = tid; x < 16 * R; x += kThreads)
         lse_s[x] = (x < N) ? lse2[((int64_t)b * Hq + h) * N + x] : 0.f;
@@ -256,54 +256,60 @@ __global__ void lse_import_kernel(const float* __restrict__ lse_in, int n, float
   if (lse_out) lse_out[x] = lse_in[x];
 }
 
-template <typename T, int R>
+template <typename TQ, typename T, int R>
 cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, const Dims& dm,
                     const float* lse_in, float2* part, float* lse2, float* scores,
                     int64_t score_stride, float* lse_out, float* syn_mass, cudaStream_t s,
-                    int* n_launch) {
+                    LaunchLog* log) {
   constexpr size_t smem = fma_smem_bytes<R>();
-  auto k1 = score_fma_kernel<T, R, false>;
-  auto k2 = score_fma_kernel<T, R, true>;
+  auto k1 = score_fma_kernel<TQ, T, R, false>;
+  auto k2 = score_fma_kernel<TQ, T, R, true>;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   const dim3 grid(t.n_chunks, dm.n_kv_heads);
   const int n_lse = t.batch * dm.n_q_heads * dm.n_pseudo;
   if (lse_in == nullptr) {
-    k1<<<grid, kThreads, smem, s>>>((const T*)q_rot, cv, t, dm, part, nullptr, nullptr, 0, nullptr);
-    ++*n_launch;
+    log->begin(kKindSweep1, s);
+    k1<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, dm, part, nullptr, nullptr, 0, nullptr);
+    log->end(s);
+    log->begin(kKindLseMerge, s);
     lse_merge_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(part, t, dm.n_q_heads, dm.n_pseudo, lse2, lse_out);
-    ++*n_launch;
+    log->end(s);
   } else {
+    log->begin(kKindLseMerge, s);
     lse_import_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(lse_in, n_lse, lse2, lse_out);
-    ++*n_launch;
+    log->end(s);
   }
-  k2<<<grid, kThreads, smem, s>>>((const T*)q_rot, cv, t, dm, nullptr, lse2, scores, score_stride, syn_mass);
-  ++*n_launch;
+  log->begin(kKindSweep2, s);
+  k2<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, dm, nullptr, lse2, scores, score_stride, syn_mass);
+  log->end(s);
   return cudaGetLastError();
 }
 
-template <typename T>
+template <typename TQ, typename T>
 cudaError_t run_fma_n(const void* q_rot, const CacheDev& cv, const SeqTable& t, const Dims& dm,
                       const float* lse_in, float2* part, float* lse2, float* scores,
                       int64_t score_stride, float* lse_out, float* syn_mass, cudaStream_t s,
-                      int* n_launch) {
+                      LaunchLog* log) {
   const int n = dm.n_pseudo;
-  if (n <= 16) return run_fma<T, 1>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
-  if (n <= 32) return run_fma<T, 2>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
-  if (n <= 64) return run_fma<T, 4>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
-  return run_fma<T, 8>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
+  if (n <= 16) return run_fma<TQ, T, 1>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  if (n <= 32) return run_fma<TQ, T, 2>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  if (n <= 64) return run_fma<TQ, T, 4>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  return run_fma<TQ, T, 8>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
 }
 
 }  // namespace
 
-cudaError_t launch_score_fma(int dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
+cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
                              const Dims& dm, const float* lse_in, float2* part, float* lse2,
                              float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
-                             cudaStream_t s, int* n_launch) {
+                             cudaStream_t s, LaunchLog* log) {
+  if (dtype == DAPQ_BF16 && q_dtype == DAPQ_BF16)
+    return run_fma_n<__nv_bfloat16, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
   if (dtype == DAPQ_BF16)
-    return run_fma_n<__nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
-  return run_fma_n<float>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, n_launch);
+    return run_fma_n<float, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  return run_fma_n<float, float>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
 }
 
 }  // namespace dapq

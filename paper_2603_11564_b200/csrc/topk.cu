@@ -122,10 +122,11 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
 }  // namespace
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
-                        const SeqTable& t, int n_kv_heads, cudaStream_t s, int* n_launch) {
+                        const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log) {
+  log->begin(kKindTopk, s);
   topk_select_kernel<<<dim3(t.batch, n_kv_heads), kTopkThreads, 0, s>>>(scores, score_stride, idx,
                                                                         idx_stride, t);
-  ++*n_launch;
+  log->end(s);
   return cudaGetLastError();
 }
 

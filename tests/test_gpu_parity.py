@@ -70,7 +70,7 @@ def _check_evict(w, data, got, ref):
 # ------------------------------------------------------------------------- dapq_rope_pseudo_q
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_rope_parity(dq, dtype):
-    w = _small(lens=(5, 131072, 4097), keep=(1, 1, 1), dtype=dtype, n_pseudo=33, rope_base=5.0e5)
+    w = _small(lens=(5, 131072, 4097), keep=(1, 1, 1), dtype=dtype, n_pseudo=33, rope_base=5.0e5, n_needles=0)
     ctx = _ctx(dq, w)
     data = gi.draw_layer(dataclasses.replace(w, prompt_lens=(8, 8, 8)), 0, "cpu")
     q = data["q_pre"].cuda()
