@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the DapQ eviction step (rotate, score, select, compact) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+One step = dapq_evict over every layer of the chosen configuration's synthetic cache
+(default: the Llama-3-8B-shaped 32k-token cache).  The metric is prompt tokens scored and
+evicted per second per layer: tokens * layers / time.  Rank 0 prints one JSON line.
+
+Under torchrun each rank runs the same workload on its own GPU: every (layer, sequence,
+KV head) is an independent unit, so the path shards with no exchange (weak scaling; NCCL
+is used only for the barrier and the max over ranks of the device time).
+
+--impl reference times the float64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from gen import inputs as gi  # noqa: E402
+
+METRIC = "prompt tokens scored+evicted/sec per layer at 1 B200; % of HBM peak"
+UNIT = "tokens/s/layer"
+
+# Recipe fallbacks, used only when MEASURED_PEAKS.json is absent.
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
+# from the ncu captures summarised under profiles/ (bytes; None = not captured for that pair).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- algorithmic work
+def layer_work(w: gi.Workload):
+    """Algorithmic bytes / flops / exps of one layer (what the method itself must move or compute)."""
+    e = 2 if w.dtype == "bf16" else 4
+    d, T, KT = w.head_dim, w.total_prompt, int(w.cu_keep[-1])
+    pairs = sum(w.n_q_heads * w.n_pseudo * (L + (w.n_pseudo + 1) / 2) for L in w.prompt_lens)   # visible (q, k) pairs
+    k_read = w.n_kv_heads * w.total_rows * d * e
+    return {
+        "k_read_bytes": k_read,
+        "score_write_bytes": 4 * w.n_kv_heads * T,
+        "gather_bytes": 4 * w.n_kv_heads * KT * d * e,           # K and V, read + write
+        "flops_per_sweep": 2.0 * pairs * d,
+        "exps_per_sweep": pairs,
+        "topk_bytes": 4 * w.n_kv_heads * T + 4 * w.n_kv_heads * KT,
+    }
+
+
+# ----------------------------------------------------------------------------- clock sampling
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, device: int):
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            self.gpu_id = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            self.gpu_id = str(device)
+        self.proc = None
+        self.out = None
+
+    def start(self):
+        self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_id}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.flush()
+        self.out.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        for line in self.out.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(self.NAMES, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.out.close()
+        os.unlink(self.out.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w": statistics.median(power) if power else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ the CPU oracle
+def oracle_sample(w: gi.Workload, layer: int = 0):
+    """Inputs of a bounded sample (whole layers, or the first KV heads of one) for the oracle."""
+    from oracle import dapq_oracle as orc
+    work = layer_work(w)
+    flops = 2 * work["flops_per_sweep"] / 2          # one float64 pass: 2 * pairs * d
+    heads = max(1, min(w.n_kv_heads, int(w.n_kv_heads * 60e9 / flops)))
+    data = gi.draw_layer(w, layer, "cpu")
+    q = data["q_pre"].double().numpy()
+    q_rot = np.stack([orc.rope_pseudo_q(q[b], w.prompt_lens[b], w.rope_base) for b in range(w.batch)])
+    gi.plant_structure(w, data, torch.from_numpy(q_rot))
+    G = w.group
+    return {"q": q[:, :heads * G], "k": data["k"][:heads].double().numpy(), "v": data["v"][:heads].double().numpy(),
+            "heads": heads}
+
+
+def time_oracle(w: gi.Workload, sample, repeats: int):
+    """Seconds per full layer, extrapolated from the sampled KV heads."""
+    from oracle import dapq_oracle as orc
+    ts = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.evict(sample["q"], sample["k"], sample["v"], w.cu_rows, w.prompt_lens, w.keep, w.rope_base)
+        ts.append((time.perf_counter() - t0) * w.n_kv_heads / sample["heads"])
+    return ts
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w: gi.Workload, budget_s: float = 20.0):
+    sample = oracle_sample(w)
+    ts = time_oracle(w, sample, 1)
+    while sum(ts) * sample["heads"] / w.n_kv_heads < budget_s / 2 and len(ts) < 4:
+        ts += time_oracle(w, sample, 1)
+    sec_per_layer = statistics.mean(ts)
+    return {"value": w.total_prompt / sec_per_layer, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"layer 0, {sample['heads']} of {w.n_kv_heads} KV heads, {len(ts)} repeat(s), "
+                      f"{sec_per_layer:.2f} s per full layer (numpy float64; BLAS threads = cores)"}
+
+
+def run_reference(args, w: gi.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = oracle_sample(w)
+    time_oracle(w, sample, args.warmup)
+    steps = args.steps
+    ts = time_oracle(w, sample, steps)
+    sec = statistics.mean(ts)
+    val = w.total_prompt / sec
+    desc = (f"each step = oracle evict of layer 0, {sample['heads']} of {w.n_kv_heads} KV heads, scaled to a full "
+            f"layer; {steps} timed step(s)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------- GPU arm
+def run_ours(args, w: gi.Workload):
+    import torch.distributed as dist
+
+    import __graft_entry__ as ge
+    import paper_2603_11564_b200 as dq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if local == 0:
+        ge.build()
+    if world > 1:
+        dist.barrier()
+    dq.load_library()
+
+    peaks = load_peaks()
+    work = layer_work(w)
+    n_layers = args.layers or w.n_layers
+    dt = w.torch_dtype()
+    KT = int(w.cu_keep[-1])
+    ctx = dq.dapq_create(w.n_q_heads, w.n_kv_heads, w.n_pseudo, w.batch, w.total_rows,
+                         dq.DAPQ_BF16 if w.dtype == "bf16" else dq.DAPQ_F32, w.rope_base, device=local)
+
+    # ---- synthetic caches, resident in HBM; structure planted with the library's own rotation
+    layers = []
+    pos = list(w.prompt_lens)
+    for l in range(n_layers):
+        data = gi.draw_layer(w, l, dev)
+        q_rot = torch.empty_like(data["q_pre"])
+        dq.dapq_rope_pseudo_q(ctx, data["q_pre"], pos, q_rot)
+        torch.cuda.synchronize()
+        gi.plant_structure(w, data, q_rot)
+        layers.append({"q": data["q_pre"], "k": data["k"], "v": data["v"],
+                       "k_out": torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt, device=dev),
+                       "v_out": torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt, device=dev)})
+    torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            dq.dapq_evict(ctx, L["q"], L["k"], L["v"], w.cu_rows, w.prompt_lens, w.keep, L["k_out"], L["v_out"])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    dq.dapq_poll_status(ctx)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    barrier()
+    n0 = dq.dapq_launch_count(ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = dq.dapq_launch_count(ctx) - n0
+    dq.dapq_poll_status(ctx)
+
+    # ---- same steps again with every kernel bracketed by CUDA events (per-kernel durations)
+    dq.dapq_profile(ctx, True)
+    for _ in range(args.steps):
+        step()
+    prof = dq.dapq_profile_read(ctx)
+    dq.dapq_profile(ctx, False)
+    clocks = sampler.stop() if sampler else None
+
+    if world > 1:
+        tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    tokens = w.total_prompt
+    value = world * tokens * n_layers / (ms_step * 1e-3)
+
+    # ---- roofline of the dominant kernel
+    kinds = {k: v for k, v in prof.items() if v[1] > 0}
+    total_prof_ms = sum(v[0] for v in kinds.values())
+    dom = max(kinds, key=lambda k: kinds[k][0])
+    dom_ms = kinds[dom][0] / kinds[dom][1]
+    if dom in ("sweep1", "sweep2"):
+        achieved = work["flops_per_sweep"] / (dom_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"]}
+    else:
+        nbytes = {"topk": work["topk_bytes"], "compact": work["gather_bytes"]}.get(dom, work["k_read_bytes"])
+        achieved = nbytes / (dom_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"]}
+    roof.update({"kernel": dom, "avg_launch_us": dom_ms * 1e3, "peak_source": peaks["source"] +
+                 (" (sustained bf16)" if roof["bound"] == "tensor" else ""),
+                 "traffic": NCU_TRAFFIC_BYTES.get((dom, w.name)),
+                 "share_of_step": kinds[dom][0] / total_prof_ms,
+                 "kernels_us": {k: round(v[0] / v[1] * 1e3, 2) for k, v in kinds.items()}})
+    layer_ms = ms_step / n_layers
+    hbm_bytes = work["k_read_bytes"] + work["score_write_bytes"] + work["gather_bytes"]
+    hbm = {"algorithmic_bytes_per_layer": hbm_bytes, "achieved_gbs": hbm_bytes / (layer_ms * 1e-3) / 1e9,
+           "frac_of_" + peaks["source"]: hbm_bytes / (layer_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        n_host = min(n_layers, 4)
+        host = []
+        for L in layers[:n_host]:
+            host.append({k: L[k].cpu().pin_memory() for k in ("q", "k", "v")})
+            host[-1]["k_out"] = torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt).pin_memory()
+            host[-1]["v_out"] = torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt).pin_memory()
+            host[-1]["idx"] = torch.empty((w.n_kv_heads, KT), dtype=torch.int32).pin_memory()
+
+        def host_step():
+            for l in range(n_layers):
+                H = host[l % n_host]
+                dq.dapq_evict_host(ctx, H["q"], H["k"], H["v"], w.cu_rows, w.prompt_lens, w.keep,
+                                   H["k_out"], H["v_out"], H["idx"])
+
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        host_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            host_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        if world > 1:
+            tt = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e2e = float(tt.item())
+        eb = 2 if w.dtype == "bf16" else 4
+        h2d = n_layers * (2 * w.n_kv_heads * w.total_rows * w.head_dim * eb + w.batch * w.n_q_heads * w.n_pseudo * w.head_dim * eb)
+        d2h = n_layers * (2 * w.n_kv_heads * KT * w.head_dim * eb + 4 * w.n_kv_heads * KT)
+        e2e = {"value": world * tokens * n_layers / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps,
+               "api": "dapq_evict_host (pinned host K/V/q in, compacted K/V + indices out, per layer)"}
+
+    dq.dapq_destroy(ctx)
+
+    base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        base = cpu_baseline(w)
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "layers": n_layers, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+                       "head_dim": w.head_dim, "batch": w.batch, "prompt_tokens": tokens, "n_pseudo": w.n_pseudo,
+                       "keep_rows": KT, "parallelism": f"independent replicas x{world}",
+                       "l2": "inputs exceed L2: every layer's K/V (%.0f MB) is distinct and read once per step"
+                             % ((2 * work["k_read_bytes"]) / 1e6)},
+            "roofline": roof, "hbm": hbm, "cpu_baseline": base, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama3_8b_32k", choices=list(gi.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the config's)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = gi.workload(args.config)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
