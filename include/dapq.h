@@ -74,6 +74,10 @@ enum { DAPQ_MAX_BATCH = 128, DAPQ_MAX_PSEUDO = 128, DAPQ_HEAD_DIM = 128 };
  * the ends of each sequence. */
 typedef enum { DAPQ_POOL_NONE = 0, DAPQ_POOL_MAX = 1, DAPQ_POOL_AVG = 2 } dapq_pool_mode;
 
+/* dapq_shape.flags.  DAPQ_FLAG_CUDA_CORE_SCORER keeps the scorer on the CUDA-core kernels
+ * (fp32 arithmetic on unrounded rotated queries) even where the tensor-core path applies. */
+typedef enum { DAPQ_FLAG_CUDA_CORE_SCORER = 1 } dapq_flags;
+
 typedef struct dapq_ctx dapq_ctx;
 
 typedef struct {
@@ -89,7 +93,7 @@ typedef struct {
   float   softmax_scale;    /* 0 -> 1/sqrt(head_dim)                              */
   int32_t pool_mode;        /* dapq_pool_mode                                     */
   int32_t pool_kernel;      /* odd window width; ignored for DAPQ_POOL_NONE       */
-  int32_t reserved;         /* must be 0                                          */
+  int32_t flags;            /* bit set of dapq_flags, normally 0                  */
 } dapq_shape;
 
 typedef struct {

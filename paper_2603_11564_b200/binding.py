@@ -21,6 +21,7 @@ DAPQ_OK, DAPQ_ERR_INVALID_ARG, DAPQ_ERR_UNSUPPORTED, DAPQ_ERR_WORKSPACE, DAPQ_ER
     DAPQ_ERR_TIMEOUT = range(6)
 DAPQ_BF16, DAPQ_F32 = 0, 1
 DAPQ_POOL_NONE, DAPQ_POOL_MAX, DAPQ_POOL_AVG = 0, 1, 2
+DAPQ_FLAG_CUDA_CORE_SCORER = 1
 _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORTED",
                  3: "DAPQ_ERR_WORKSPACE", 4: "DAPQ_ERR_CUDA", 5: "DAPQ_ERR_TIMEOUT"}
 
@@ -40,7 +41,7 @@ class dapq_shape(C.Structure):
                 ("n_pseudo", C.c_int32), ("max_batch", C.c_int32), ("dtype", C.c_int32),
                 ("max_total_rows", C.c_int64), ("rope_base", C.c_double),
                 ("inv_freq_host", C.POINTER(C.c_double)), ("softmax_scale", C.c_float),
-                ("pool_mode", C.c_int32), ("pool_kernel", C.c_int32), ("reserved", C.c_int32)]
+                ("pool_mode", C.c_int32), ("pool_kernel", C.c_int32), ("flags", C.c_int32)]
 
 
 class dapq_cache_view(C.Structure):
@@ -134,12 +135,12 @@ def _view(k: torch.Tensor, v: Optional[torch.Tensor], cu_rows, prompt_len):
 def dapq_create(n_q_heads: int, n_kv_heads: int, n_pseudo: int, max_batch: int, max_total_rows: int,
                 dtype: int, rope_base: float, head_dim: int = 128, softmax_scale: float = 0.0,
                 inv_freq: Optional[Sequence[float]] = None, pool_mode: int = DAPQ_POOL_NONE,
-                pool_kernel: int = 1, device: int = 0):
+                pool_kernel: int = 1, flags: int = 0, device: int = 0):
     lib = load_library()
     sh = dapq_shape(n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim, n_pseudo=n_pseudo,
                     max_batch=max_batch, dtype=dtype, max_total_rows=max_total_rows,
                     rope_base=rope_base, softmax_scale=softmax_scale, pool_mode=pool_mode,
-                    pool_kernel=pool_kernel, reserved=0)
+                    pool_kernel=pool_kernel, flags=flags)
     if inv_freq is not None:
         arr = (C.c_double * len(inv_freq))(*[float(x) for x in inv_freq])
         sh.inv_freq_host = C.cast(arr, C.POINTER(C.c_double))

@@ -17,7 +17,9 @@ struct dapq_ctx {
   dapq_shape shape{};
   Dims dims{};
   int elem_bytes = 2;
+  int n_sm = 148;
   int64_t max_chunks = 0;
+  int64_t q_rows_max = 0;        // max_batch * H_q * N
   // device workspace
   double* inv_freq = nullptr;    // [d/2]
   int* status = nullptr;         // device status word
@@ -148,7 +150,6 @@ dapq_status build_table(dapq_ctx* ctx, int32_t batch, const int32_t* cu_rows, co
     if (pos_start && pos_start[b] < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "pos_start[%d] is negative", b);
     t->cu_prompt[b] = (int32_t)prompt;
     t->cu_keep[b] = (int32_t)keep;
-    t->cu_chunk[b] = (int32_t)chunks;
     rows += L + sh.n_pseudo;
     prompt += L;
     keep += kb;
@@ -156,8 +157,6 @@ dapq_status build_table(dapq_ctx* ctx, int32_t batch, const int32_t* cu_rows, co
   }
   t->cu_prompt[batch] = (int32_t)prompt;
   t->cu_keep[batch] = (int32_t)keep;
-  t->cu_chunk[batch] = (int32_t)chunks;
-  t->n_chunks = (int32_t)chunks;
   const int64_t last_row = cu_rows ? cu_rows[batch] : rows;
   if ((prompt_len || cu_prompt) && (last_row > sh.max_total_rows || chunks > ctx->max_chunks))
     return fail(ctx, DAPQ_ERR_WORKSPACE, "%lld cache rows exceed max_total_rows %lld",
@@ -186,6 +185,22 @@ dapq_status check_view(dapq_ctx* ctx, const dapq_cache_view* cv, bool need_v, bo
   out->k_row_stride = cv->k_row_stride;
   out->v_head_stride = cv->v_head_stride;
   out->v_row_stride = cv->v_row_stride;
+  return DAPQ_OK;
+}
+
+// The tensor-core scorer takes bf16 caches whose query block is at least half an MMA tile high;
+// everything else (fp32 storage, tiny windows, views TMA cannot describe, syn_mass requests)
+// goes to the CUDA-core scorer.
+bool wants_umma(const dapq_ctx* ctx) {
+  return ctx->shape.dtype == DAPQ_BF16 && !(ctx->shape.flags & DAPQ_FLAG_CUDA_CORE_SCORER) &&
+         ctx->dims.group * ctx->dims.n_pseudo >= 64;
+}
+
+dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& t, const float* lse_in,
+                           float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
+  cudaError_t e = launch_score_umma(plan, t, ctx->dims, lse_in, ctx->part, ctx->lse2, scores, score_stride,
+                                    lse_out, ctx->status, s, &ctx->log);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels");
   return DAPQ_OK;
 }
 
@@ -222,7 +237,7 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   if (sh->max_batch > kMaxBatch || sh->max_total_rows > 0x7fffffffLL)
     return bail(DAPQ_ERR_UNSUPPORTED, "max_batch > 128 or max_total_rows >= 2^31");
   if (sh->dtype != DAPQ_BF16 && sh->dtype != DAPQ_F32) return bail(DAPQ_ERR_INVALID_ARG, "unknown dtype");
-  if (sh->reserved != 0) return bail(DAPQ_ERR_INVALID_ARG, "reserved must be 0");
+  if (sh->flags & ~DAPQ_FLAG_CUDA_CORE_SCORER) return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
   if (sh->pool_mode != DAPQ_POOL_NONE) return bail(DAPQ_ERR_UNSUPPORTED, "pooling is not available");
   if (!sh->inv_freq_host && !(sh->rope_base > 0.0)) return bail(DAPQ_ERR_INVALID_ARG, "rope_base must be > 0");
   if (!(sh->softmax_scale >= 0.f)) return bail(DAPQ_ERR_INVALID_ARG, "softmax_scale must be >= 0");
@@ -244,14 +259,20 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   double freq[kHeadDim / 2];
   for (int c = 0; c < kHeadDim / 2; ++c)
     freq[c] = sh->inv_freq_host ? sh->inv_freq_host[c] : pow(sh->rope_base, -2.0 * c / (double)kHeadDim);
+  if (cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || ctx->n_sm < 1)
+    return bail(DAPQ_ERR_CUDA, "cannot query the device");
   const size_t hq_n = (size_t)sh->n_q_heads * sh->n_pseudo;
+  ctx->q_rows_max = (int64_t)sh->max_batch * hq_n;
+  size_t part_elems = (size_t)ctx->max_chunks * hq_n;
+  const size_t part_umma = (size_t)umma_part_elems(sh->max_batch, sh->n_q_heads, sh->n_kv_heads, sh->n_pseudo);
+  if (part_umma > part_elems) part_elems = part_umma;
   const size_t rows = (size_t)sh->max_total_rows;
   bool ok = true;
   ok = ok && cudaMalloc(&ctx->inv_freq, sizeof(freq)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->status, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->q_rot, (size_t)sh->max_batch * hq_n * kHeadDim * sizeof(float)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->part, (size_t)ctx->max_chunks * hq_n * sizeof(float2)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->lse2, (size_t)sh->max_batch * hq_n * sizeof(float)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->part, part_elems * sizeof(float2)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->lse2, ((size_t)sh->max_batch * hq_n + 32) * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->scores, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->idx, (size_t)sh->n_kv_heads * rows * sizeof(int32_t)) == cudaSuccess;
   ok = ok && cudaMemcpy(ctx->inv_freq, freq, sizeof(freq), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -331,7 +352,7 @@ dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* 
   dapq_status st = build_table(ctx, batch, nullptr, nullptr, nullptr, nullptr, pos_start_host, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  cudaError_t e = launch_rope(ctx->shape.dtype, ctx->shape.dtype, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &ctx->log);
+  cudaError_t e = launch_rope(ctx->shape.dtype, ctx->shape.dtype, 0, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
   return DAPQ_OK;
 }
@@ -348,6 +369,11 @@ dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* 
   st = build_table(ctx, cache->batch, cache->cu_rows_host, cache->prompt_len_host, nullptr, nullptr, nullptr, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
+  if (wants_umma(ctx) && !syn_mass) {
+    UmmaPlan plan;
+    if (umma_plan(q_rot, 0, 0, cd, t, ctx->dims, ctx->n_sm, &plan))
+      return run_score_umma(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, (cudaStream_t)stream);
+  }
   return run_score(ctx, ctx->shape.dtype, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
 }
 
@@ -398,13 +424,24 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)stream;
-  // the CUDA-core scorer reads the rotated queries unrounded (fp32)
-  cudaError_t e = launch_rope(ctx->shape.dtype, DAPQ_F32, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &ctx->log);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
   float* scores = scores_out ? scores_out : ctx->scores;
   int32_t* idx = idx_out ? idx_out : ctx->idx;
   const int64_t score_stride = t.cu_prompt[t.batch], idx_stride = t.cu_keep[t.batch];
-  st = run_score(ctx, DAPQ_F32, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
+  UmmaPlan plan;
+  const int64_t lo_rows = ctx->q_rows_max;
+  cudaError_t e;
+  if (wants_umma(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {
+    // tensor-core scorer: rotated queries as a bf16 pair hi + lo (two MMAs per k-step)
+    e = launch_rope(ctx->shape.dtype, kRopeOutSplitBf16, lo_rows * kHeadDim, q_pre, ctx->q_rot, ctx->inv_freq, t,
+                    ctx->dims, s, &ctx->log);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
+    st = run_score_umma(ctx, plan, t, nullptr, scores, score_stride, nullptr, s);
+  } else {
+    // CUDA-core scorer: reads the rotated queries unrounded (fp32)
+    e = launch_rope(ctx->shape.dtype, kRopeOutF32, 0, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &ctx->log);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
+    st = run_score(ctx, DAPQ_F32, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
+  }
   if (st != DAPQ_OK) return st;
   e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");

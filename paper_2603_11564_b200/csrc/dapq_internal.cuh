@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libdapq (not installed).
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -17,15 +18,22 @@ constexpr int kChunkKeys = 512;              // prompt keys per work chunk of th
 // be copied to the device, so a call adds no copy nodes to a stream).
 struct SeqTable {
   int32_t batch;
-  int32_t n_chunks;                 // sum_b (ceil(L_b / kChunkKeys) + 1)
   int32_t cu_rows[kMaxBatch + 1];   // first cache row of sequence b
   int32_t cu_prompt[kMaxBatch + 1]; // first score column of sequence b
   int32_t cu_keep[kMaxBatch + 1];   // first output row of sequence b (K_b clamped to L_b)
-  int32_t cu_chunk[kMaxBatch + 1];  // first work chunk of sequence b; its last chunk holds the
-                                    // N synthetic rows, the others kChunkKeys prompt rows each
   int32_t prompt_len[kMaxBatch];    // L_b
   int32_t pos_start[kMaxBatch];     // position of pseudo query 0
 };
+
+// How the score sweeps cut the sequences into work chunks (one CTA per chunk and KV head).
+//   CUDA-core path:   chunks of kChunkKeys prompt keys, then one chunk with the N synthetic rows;
+//   tensor-core path: chunks of chunk_tiles 128-row tiles over the rows [0, L_b + N).
+struct ChunkTable {
+  int32_t chunk_tiles;
+  int32_t n_chunks;
+  int32_t cu_chunk[kMaxBatch + 1];  // first chunk of sequence b
+};
+constexpr int kUmmaMaxChunks = 256;  // the tensor-core planner never makes more chunks than max_batch + this
 
 struct CacheDev {
   const void* k;
@@ -40,6 +48,9 @@ struct Dims {
 
 // Device status word bits (set by kernels, read by dapq_poll_status).
 enum : int { kStatusTimeout = 1, kStatusBadIndex = 2 };
+
+// Output formats of the rotation kernel.
+enum : int { kRopeOutBf16 = DAPQ_BF16, kRopeOutF32 = DAPQ_F32, kRopeOutSplitBf16 = 2 };
 
 __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
   // largest b in [0, n) with cu[b] <= x
@@ -66,9 +77,10 @@ struct LaunchLog {
 };
 
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------
-// q_pre has element type `dtype`; q_rot is written as `out_dtype` (fp32 keeps the rotated
-// queries unrounded for the CUDA-core scorer).
-cudaError_t launch_rope(int dtype, int out_dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
+// q_pre has element type `dtype`; q_rot is written as `out_mode`: bf16, fp32 (unrounded, for
+// the CUDA-core scorer) or a bf16 pair hi + lo with lo = bf16(q - hi) stored `lo_offset`
+// elements after hi (for the tensor-core scorer).
+cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* q_pre, void* q_rot, const double* inv_freq_dev,
                         const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log);
 
 // Generic CUDA-core scorer (any N <= 128, both dtypes).
@@ -78,6 +90,23 @@ cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const Ca
                              const Dims& dm, const float* lse_in, float2* part, float* lse2,
                              float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
                              cudaStream_t s, LaunchLog* log);
+
+// Tensor-core scorer (bf16 caches).  umma_plan encodes the TMA descriptors and cuts the work;
+// it returns false when the view cannot be described to TMA (the caller then takes the
+// CUDA-core path).  q_hi: [B*H_q*N, d] bf16; with has_lo the low-order parts follow
+// lo_row_offset rows later in the same allocation.
+struct UmmaPlan {
+  CUtensorMap tm_k, tm_q;
+  ChunkTable ct;
+  int32_t has_lo;
+  int64_t lo_row_offset;
+};
+bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheDev& cv, const SeqTable& t,
+               const Dims& dm, int n_sm, UmmaPlan* plan);
+int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo);
+cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
+                              float2* part, float* lse2, float* scores, int64_t score_stride, float* lse_out,
+                              int* status, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log);

@@ -22,11 +22,12 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(
   return __double2bfloat16(x);
 }
 
-template <typename T, typename TO>
+// kSplit: TO is bf16 and the rounding residual is stored as a second bf16 lo_offset elements on.
+template <typename T, typename TO, bool kSplit>
 __global__ void __launch_bounds__(kHeadDim / 2)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
-                     int n_q_heads, int n_pseudo) {
+                     int n_q_heads, int n_pseudo, int64_t lo_offset) {
   const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   constexpr int half = kHeadDim / 2;
   const double ang = (double)(t.pos_start[b] + i) * inv_freq[c];
@@ -36,26 +37,36 @@ rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
     const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
     const double lo = to_double<T>(q_pre[base + c]);
     const double hi = to_double<T>(q_pre[base + c + half]);
-    q_rot[base + c] = from_double<TO>(lo * cs - hi * sn);
-    q_rot[base + c + half] = from_double<TO>(hi * cs + lo * sn);
+    const double r0 = lo * cs - hi * sn, r1 = hi * cs + lo * sn;
+    const TO h0 = from_double<TO>(r0), h1 = from_double<TO>(r1);
+    q_rot[base + c] = h0;
+    q_rot[base + c + half] = h1;
+    if (kSplit) {
+      q_rot[lo_offset + base + c] = from_double<TO>(r0 - to_double<TO>(h0));
+      q_rot[lo_offset + base + c + half] = from_double<TO>(r1 - to_double<TO>(h1));
+    }
   }
 }
 
 }  // namespace
 
-cudaError_t launch_rope(int dtype, int out_dtype, const void* q_pre, void* q_rot, const double* inv_freq_dev,
-                        const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log) {
+cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* q_pre, void* q_rot,
+                        const double* inv_freq_dev, const SeqTable& t, const Dims& dm, cudaStream_t s,
+                        LaunchLog* log) {
   log->begin(kKindRope, s);
   dim3 grid(dm.n_pseudo, t.batch), block(kHeadDim / 2);
-  if (dtype == DAPQ_BF16 && out_dtype == DAPQ_BF16) {
-    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, block, 0, s>>>(
-        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+  if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
+    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true><<<grid, block, 0, s>>>(
+        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset);
+  } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
+    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false><<<grid, block, 0, s>>>(
+        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   } else if (dtype == DAPQ_BF16) {
-    rope_pseudo_q_kernel<__nv_bfloat16, float><<<grid, block, 0, s>>>(
-        (const __nv_bfloat16*)q_pre, (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+    rope_pseudo_q_kernel<__nv_bfloat16, float, false><<<grid, block, 0, s>>>(
+        (const __nv_bfloat16*)q_pre, (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   } else {
-    rope_pseudo_q_kernel<float, float><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
-                                                              inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo);
+    rope_pseudo_q_kernel<float, float, false><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
+                                                                     inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   }
   log->end(s);
   return cudaGetLastError();

@@ -76,7 +76,7 @@ constexpr size_t fma_smem_bytes() {
 template <typename TQ, typename T, int R, bool kSweep2>
 __global__ void __launch_bounds__(kThreads)
 score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_constant__ SeqTable t,
-                 const Dims dm, float2* __restrict__ part, const float* __restrict__ lse2,
+                 const __grid_constant__ ChunkTable ct, const Dims dm, float2* __restrict__ part, const float* __restrict__ lse2,
                  float* __restrict__ scores, int64_t score_stride, float* __restrict__ syn_mass) {
   extern __shared__ __align__(16) float smem[];
   float* Qs = smem;                          // [16 R][kPad]
@@ -86,10 +86,10 @@ score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_c
   float* lse_s = colacc + kChunkKeys;        // [16 R]
 
   const int chunk = blockIdx.x, kvh = blockIdx.y, tid = threadIdx.x;
-  const int b = find_segment(t.cu_chunk, t.batch, chunk);
-  const int c = chunk - t.cu_chunk[b];
+  const int b = find_segment(ct.cu_chunk, t.batch, chunk);
+  const int c = chunk - ct.cu_chunk[b];
   const int L = t.prompt_len[b], N = dm.n_pseudo, G = dm.group, Hq = dm.n_q_heads;
-  const bool syn = (c == t.cu_chunk[b + 1] - t.cu_chunk[b] - 1);
+  const bool syn = (c == ct.cu_chunk[b + 1] - ct.cu_chunk[b] - 1);
   const int key_begin = syn ? L : c * kChunkKeys;
   const int key_end = syn ? L + N : min(L, key_begin + kChunkKeys);
   if (kSweep2 && syn && syn_mass == nullptr) return;
@@ -228,17 +228,17 @@ score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_c
 
 // Merge the per-chunk (max, sum) partials of one pseudo query into its base-2 log-sum-exp.
 __global__ void lse_merge_kernel(const float2* __restrict__ part, const __grid_constant__ SeqTable t,
-                                 int n_q_heads, int n_pseudo, float* __restrict__ lse2,
+                                 const __grid_constant__ ChunkTable ct, int n_q_heads, int n_pseudo, float* __restrict__ lse2,
                                  float* __restrict__ lse_out) {
   const int x = blockIdx.x * blockDim.x + threadIdx.x;
   const int per_seq = n_q_heads * n_pseudo;
   if (x >= t.batch * per_seq) return;
   const int b = x / per_seq, hi = x % per_seq;
   float mx = -CUDART_INF_F;
-  for (int c = t.cu_chunk[b]; c < t.cu_chunk[b + 1]; ++c)
+  for (int c = ct.cu_chunk[b]; c < ct.cu_chunk[b + 1]; ++c)
     mx = fmaxf(mx, part[(int64_t)c * per_seq + hi].x);
   float z = 0.f;
-  for (int c = t.cu_chunk[b]; c < t.cu_chunk[b + 1]; ++c) {
+  for (int c = ct.cu_chunk[b]; c < ct.cu_chunk[b + 1]; ++c) {
     const float2 p = part[(int64_t)c * per_seq + hi];
     z += p.y * exp2f(p.x - mx);
   }
@@ -267,14 +267,23 @@ cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, co
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  const dim3 grid(t.n_chunks, dm.n_kv_heads);
+  ChunkTable ct;
+  ct.chunk_tiles = 0;
+  int32_t n_chunks = 0;
+  for (int b = 0; b < t.batch; ++b) {
+    ct.cu_chunk[b] = n_chunks;
+    n_chunks += (t.prompt_len[b] + kChunkKeys - 1) / kChunkKeys + 1;
+  }
+  ct.cu_chunk[t.batch] = n_chunks;
+  ct.n_chunks = n_chunks;
+  const dim3 grid(n_chunks, dm.n_kv_heads);
   const int n_lse = t.batch * dm.n_q_heads * dm.n_pseudo;
   if (lse_in == nullptr) {
     log->begin(kKindSweep1, s);
-    k1<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, dm, part, nullptr, nullptr, 0, nullptr);
+    k1<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, ct, dm, part, nullptr, nullptr, 0, nullptr);
     log->end(s);
     log->begin(kKindLseMerge, s);
-    lse_merge_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(part, t, dm.n_q_heads, dm.n_pseudo, lse2, lse_out);
+    lse_merge_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(part, t, ct, dm.n_q_heads, dm.n_pseudo, lse2, lse_out);
     log->end(s);
   } else {
     log->begin(kKindLseMerge, s);
@@ -282,7 +291,7 @@ cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, co
     log->end(s);
   }
   log->begin(kKindSweep2, s);
-  k2<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, dm, nullptr, lse2, scores, score_stride, syn_mass);
+  k2<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, ct, dm, nullptr, lse2, scores, score_stride, syn_mass);
   log->end(s);
   return cudaGetLastError();
 }

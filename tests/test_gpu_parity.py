@@ -112,28 +112,35 @@ def test_score_parity(dq, dtype, hq, hkv, n, lens):
     scores = torch.empty((hkv, w.total_prompt), dtype=torch.float32, device="cuda")
     lse = torch.empty((B, hq, n), dtype=torch.float32, device="cuda")
     syn = torch.empty((B, hq), dtype=torch.float32, device="cuda")
-    dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, lse_out=lse, syn_mass=syn)
-    dq.dapq_poll_status(ctx)
-    first = scores.clone()
-    # bit-identical when repeated (fixed reduction order, no float atomics)
-    dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, lse_out=lse, syn_mass=syn)
-    torch.cuda.synchronize()
-    assert torch.equal(first, scores)
-    got = scores.cpu().double().numpy()
     k64 = util.to_f64(data["k"])
-    for b in range(B):
-        r0, L = int(w.cu_rows[b]), lens[b]
-        ref = orc.score_sequence(util.to_f64(q_rot[b]), k64[:, r0:r0 + L + n], L, w.group)
-        util.assert_scores_close(got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]], ref["scores"], f"b={b}")
-        np.testing.assert_allclose(lse[b].cpu().numpy(), ref["lse"], rtol=0, atol=2e-3)
-        np.testing.assert_allclose(syn[b].cpu().numpy(), ref["syn_mass"], rtol=2e-3, atol=1e-6)
-        # mass conservation on the GPU's own numbers: sum_j scores + sum_g syn = G * N
-        tot = got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]].sum(axis=1) + syn[b].cpu().double().numpy().reshape(hkv, -1).sum(axis=1)
-        np.testing.assert_allclose(tot, np.full(hkv, w.group * n), rtol=1e-4)
+    refs = [orc.score_sequence(util.to_f64(q_rot[b]), k64[:, int(w.cu_rows[b]):int(w.cu_rows[b + 1])], lens[b], w.group)
+            for b in range(B)]
+    # without syn_mass the bf16 shapes with G*N >= 64 run on the tensor cores; asking for
+    # syn_mass routes the same call through the CUDA-core kernels
+    for want_syn in (False, True):
+        scores.fill_(-1.0)
+        lse.fill_(0.0)
+        kw = dict(lse_out=lse, syn_mass=syn) if want_syn else dict(lse_out=lse)
+        dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, **kw)
+        dq.dapq_poll_status(ctx)
+        first = scores.clone()
+        # bit-identical when repeated (fixed reduction order, no float atomics)
+        dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores, **kw)
+        dq.dapq_poll_status(ctx)
+        assert torch.equal(first, scores)
+        got = scores.cpu().double().numpy()
+        for b in range(B):
+            ref = refs[b]
+            util.assert_scores_close(got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]], ref["scores"], f"b={b} syn={want_syn}")
+            np.testing.assert_allclose(lse[b].cpu().numpy(), ref["lse"], rtol=0, atol=2e-3)
+            if want_syn:
+                np.testing.assert_allclose(syn[b].cpu().numpy(), ref["syn_mass"], rtol=2e-3, atol=1e-6)
+                # mass conservation on the GPU's own numbers: sum_j scores + sum_g syn = G * N
+                tot = (got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]].sum(axis=1)
+                       + syn[b].cpu().double().numpy().reshape(hkv, -1).sum(axis=1))
+                np.testing.assert_allclose(tot, np.full(hkv, w.group * n), rtol=1e-4)
     # the caller's own log-sum-exp (from the oracle) replaces the first sweep
-    lse_ref = torch.from_numpy(np.stack([
-        orc.score_sequence(util.to_f64(q_rot[b]), k64[:, int(w.cu_rows[b]):int(w.cu_rows[b + 1])], lens[b], w.group)["lse"]
-        for b in range(B)])).float().cuda()
+    lse_ref = torch.from_numpy(np.stack([refs[b]["lse"] for b in range(B)])).float().cuda()
     scores2 = torch.empty_like(scores)
     dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores2, lse_in=lse_ref)
     torch.cuda.synchronize()
@@ -225,12 +232,15 @@ def test_evict_tiny_config_in_full(dq):
     _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
 
 
+@pytest.mark.parametrize("cuda_core", [False, True])
 @pytest.mark.parametrize("name,scale", [("llama3_8b_32k", 16), ("qwen25_7b_128k", 64), ("batched_serving", 16),
                                         ("llama3_70b_128k", 64)])
-def test_evict_scaled_configs(dq, name, scale):
+def test_evict_scaled_configs(dq, name, scale, cuda_core):
     w = gi.scaled_down(name, scale, n_layers=1)
     data = util.make_case(w)
-    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+    ctx = _ctx(dq, w, flags=dq.DAPQ_FLAG_CUDA_CORE_SCORER if cuda_core else 0)
+    _check_evict(w, data, _gpu_evict(dq, w, data, ctx), util.oracle_evict(w, data))
+    dq.dapq_destroy(ctx)
 
 
 def test_evict_edge_shapes(dq):
