@@ -198,7 +198,7 @@ bool wants_umma(const dapq_ctx* ctx) {
 
 dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& t, const float* lse_in,
                            float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
-  cudaError_t e = launch_score_umma(plan, t, ctx->dims, lse_in, ctx->part, ctx->lse2, scores, score_stride,
+  cudaError_t e = launch_score_umma(plan, t, ctx->dims, lse_in, ctx->part, scores, score_stride,
                                     lse_out, ctx->status, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels");
   return DAPQ_OK;

@@ -105,7 +105,7 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
                const Dims& dm, int n_sm, UmmaPlan* plan);
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo);
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
-                              float2* part, float* lse2, float* scores, int64_t score_stride, float* lse_out,
+                              float2* part, float* scores, int64_t score_stride, float* lse_out,
                               int* status, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,

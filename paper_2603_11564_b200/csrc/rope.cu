@@ -2,14 +2,18 @@
 // tokens take positions L_p .. L_p+N-1, so their queries carry the positional encodings of
 // the first N decoding steps).
 //
-// One CTA per (pseudo query i, sequence b); thread c owns the channel pair (c, c + d/2).
-// The angle pos * theta_c is formed and reduced in double precision: at positions near
-// 131k a float angle has only ~7 fractional bits, which alone would cost half of the
-// scorer's error budget.  The table is tiny (B*N*64 sincos), so this costs nothing.
+// Grid (pseudo query i, sequence b, block of query heads); thread (c, hy) owns the channel
+// pair (c, c + d/2) of one head.  The angle pos * theta_c is formed and reduced in double
+// precision: at positions near 131k a float angle has only ~7 fractional bits, which alone
+// would cost half of the scorer's error budget.  Each thread evaluates its own sincos (the
+// table is tiny: B*N*64 angles), so no thread waits on another and the launch is one short
+// wave of independent loads and stores.
 #include "dapq_internal.cuh"
 
 namespace dapq {
 namespace {
+
+constexpr int kHeadsPerBlock = 8;
 
 template <typename T> __device__ __forceinline__ double to_double(T x);
 template <> __device__ __forceinline__ double to_double<float>(float x) { return (double)x; }
@@ -24,27 +28,27 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(
 
 // kSplit: TO is bf16 and the rounding residual is stored as a second bf16 lo_offset elements on.
 template <typename T, typename TO, bool kSplit>
-__global__ void __launch_bounds__(kHeadDim / 2)
+__global__ void __launch_bounds__(kHeadDim / 2 * kHeadsPerBlock)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
                      int n_q_heads, int n_pseudo, int64_t lo_offset) {
   const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  const int h = blockIdx.z * kHeadsPerBlock + threadIdx.y;
+  if (h >= n_q_heads) return;
   constexpr int half = kHeadDim / 2;
+  const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
+  const double lo = to_double<T>(q_pre[base + c]);
+  const double hi = to_double<T>(q_pre[base + c + half]);
   const double ang = (double)(t.pos_start[b] + i) * inv_freq[c];
   double sn, cs;
   sincos(ang, &sn, &cs);
-  for (int h = 0; h < n_q_heads; ++h) {
-    const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
-    const double lo = to_double<T>(q_pre[base + c]);
-    const double hi = to_double<T>(q_pre[base + c + half]);
-    const double r0 = lo * cs - hi * sn, r1 = hi * cs + lo * sn;
-    const TO h0 = from_double<TO>(r0), h1 = from_double<TO>(r1);
-    q_rot[base + c] = h0;
-    q_rot[base + c + half] = h1;
-    if (kSplit) {
-      q_rot[lo_offset + base + c] = from_double<TO>(r0 - to_double<TO>(h0));
-      q_rot[lo_offset + base + c + half] = from_double<TO>(r1 - to_double<TO>(h1));
-    }
+  const double r0 = lo * cs - hi * sn, r1 = hi * cs + lo * sn;
+  const TO h0 = from_double<TO>(r0), h1 = from_double<TO>(r1);
+  q_rot[base + c] = h0;
+  q_rot[base + c + half] = h1;
+  if (kSplit) {
+    q_rot[lo_offset + base + c] = from_double<TO>(r0 - to_double<TO>(h0));
+    q_rot[lo_offset + base + c + half] = from_double<TO>(r1 - to_double<TO>(h1));
   }
 }
 
@@ -54,7 +58,8 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
                         const double* inv_freq_dev, const SeqTable& t, const Dims& dm, cudaStream_t s,
                         LaunchLog* log) {
   log->begin(kKindRope, s);
-  dim3 grid(dm.n_pseudo, t.batch), block(kHeadDim / 2);
+  dim3 grid(dm.n_pseudo, t.batch, (dm.n_q_heads + kHeadsPerBlock - 1) / kHeadsPerBlock);
+  dim3 block(kHeadDim / 2, kHeadsPerBlock);
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
     rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true><<<grid, block, 0, s>>>(
         (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset);

@@ -11,17 +11,22 @@
 // Two sweeps (column sums of a row-normalised matrix need every row's normaliser first):
 //   sweep 1   D[query, key] = Q_blk K_tile^T   queries on TMEM lanes: each thread owns one
 //             pseudo query and keeps its running max / sum of exp -> partials per chunk;
-//   sweep 2   D[key, query] = K_tile Q_grp^T   keys on TMEM lanes: each thread owns one key
+//   sweep 2   D[key, query] = K_tile Q_blk^T   keys on TMEM lanes: each thread owns one key
 //             and sums exp2(s - lse_i) over the query columns -> scores, coalesced store.
+//             Its epilogue threads first merge the partials of sweep 1 into the log-sum-exp
+//             of the resident query rows (kept in shared memory), so no kernel runs between
+//             the sweeps.
 // The rotated queries are used as a bf16 pair (hi + lo, lo = bf16(q - hi)): two MMAs per
 // k-step with the same K tile.  A single bf16 rounding of q would put the per-token scores
 // of caches with outlier channels outside the 2e-3 tolerance.
 //
 // CTA = (chunk of 128-key tiles, KV head); 10 warps: warp 0 issues TMA loads (K tiles
 // through a 3-stage ring, the query group once), warp 1 issues the MMAs and owns tensor
-// memory, warps 2-9 are two epilogue groups (4 warps = 128 TMEM lanes each) that take
-// alternate accumulators.  Every mbarrier wait is bounded: after ~1 s the CTA raises the
-// timeout status, drains and returns normally.
+// memory, warps 2-9 are two epilogue groups (4 warps = 128 TMEM lanes each).  An accumulator
+// job is a [128 x 128] fp32 block; four fit in tensor memory, so the MMA warp runs up to
+// four jobs ahead of the epilogue, which reads each block in 32-column pieces with the next
+// piece's load in flight while the current one is exponentiated.  Every mbarrier wait is
+// bounded: after ~1 s the CTA raises the timeout status, drains and returns normally.
 #include <cuda.h>
 #include <math_constants.h>
 
@@ -48,7 +53,8 @@ struct Smem {
   static constexpr int k = q_lo + kQBytes;
   static constexpr int bars = k + kStages * kTileBytes;
   // barriers: k_full[3], k_empty[3], acc_full[4], acc_empty[4], q_full, q_empty  (16 x 8 B)
-  static constexpr int tmem_ptr = bars + 16 * 8;
+  static constexpr int lse = bars + 16 * 8;          // [256] floats
+  static constexpr int tmem_ptr = lse + kGroupRows * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -132,26 +138,50 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Three-input maximum (one instruction on sm_100).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// Wait for this thread's outstanding tensor-memory loads.  The registers of the load being
+// waited for are passed through so that no use of them can be scheduled above the wait.
+__device__ __forceinline__ void tmem_ld_wait_for(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
+}
+// Barrier among the 8 epilogue warps only (the producer warps never join it).
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
 struct UmmaArgs {
   int32_t n_pseudo, group, n_q_heads, n_kv_heads;
   int32_t rows_total;        // G * N
   int32_t n_qgroups;         // ceil(rows_total / 256)
   int32_t has_lo;            // the query operand carries a low-order bf16 part
   int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
-  int32_t n_lse;             // B * H_q * N (entries of lse2; 32 floats of slack follow)
   float scale_log2e;
-  float2* part;              // [n_chunks, H_kv, 2, n_qgroups * 256]
-  const float* lse2;         // [B, H_q, N]
+  float2* part;              // [n_chunks, H_kv, 2, n_qgroups * 256] (running max, sum) in base 2
+  const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
+  float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
   float* scores;
   int64_t score_stride;
   int* status;
 };
+
+// One accumulator job is a [128 x 128] fp32 block in tensor memory (4 of them fit):
+//   sweep 1: 128 pseudo queries (lanes) x 128 keys (columns);
+//   sweep 2: 128 keys (lanes) x 128 pseudo queries (columns).
+constexpr int kAccBufs = 4;
+constexpr int kAccCols = kTmemCols / kAccBufs;
 
 template <bool kSweep2>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -183,8 +213,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const uint32_t q_full = bar0 + 8u * 14, q_empty = bar0 + 8u * 15;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Smem::tmem_ptr);
-  constexpr int kAccBufs = kSweep2 ? 2 : 4;                     // 256 / 128 TMEM columns each
-  constexpr int kAccCols = kTmemCols / kAccBufs;
+  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] base-2 lse of the resident query group
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
@@ -248,29 +277,29 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
         const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
         const int mb = (rows_g + 127) / 128;
-        const int n2 = (rows_g + 31) & ~31;                     // sweep 2: query columns per MMA
         ok = mbar_wait(q_full, qg & 1, abort_flag, a.status);
         for (int ti = 0; ti < nt && ok; ++ti, ++li) {
           const int s = li % kStages;
           ok = mbar_wait(k_full(s), (li / kStages) & 1, abort_flag, a.status);
           if (!ok) break;
           const uint32_t kaddr = sbase + Smem::k + s * kTileBytes;
-          const int n_jobs = kSweep2 ? 1 : mb;
-          for (int m = 0; m < n_jobs && ok; ++m, ++job) {
+          for (int m = 0; m < mb && ok; ++m, ++job) {
             const int buf = job % kAccBufs;
             if (job >= kAccBufs) ok = mbar_wait(acc_empty(buf), ((job / kAccBufs) - 1) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d = tmem_base + buf * kAccCols;
+            // sweep 2: only the query columns that exist (rounded up to the MMA's N granule of 16)
+            const int n2 = (min(128, rows_g - m * 128) + 15) & ~15;
             const uint32_t idesc = kSweep2 ? umma_idesc(128, n2) : umma_idesc(128, kTileKeys);
             uint32_t accum = 0;
             for (int part = 0; part < (a.has_lo ? 2 : 1); ++part) {
-              const uint32_t qaddr = sbase + (part ? Smem::q_lo : Smem::q_hi);
+              const uint32_t qaddr = sbase + (part ? Smem::q_lo : Smem::q_hi) + m * 128 * 128;
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
                 const int half = ks >> 2, kk = ks & 3;
                 const uint64_t kd = umma_desc(kaddr + half * kHalfBytesK + kk * 32);
-                const uint64_t qd = umma_desc(qaddr + half * kHalfBytesQ + (kSweep2 ? 0 : m * 128 * 128) + kk * 32);
+                const uint64_t qd = umma_desc(qaddr + half * kHalfBytesQ + kk * 32);
                 if (kSweep2) umma(d, kd, qd, idesc, accum); else umma(d, qd, kd, idesc, accum);
                 accum = 1;
               }
@@ -291,59 +320,90 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const float c = a.scale_log2e;
     int job = 0;
     bool ok = true;
-    for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+    // (an aborting group still walks every query group: the other group waits for it at the barriers)
+    for (int qg = 0; qg < a.n_qgroups && (ok || kSweep2); ++qg) {
       const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
       const int mb = (rows_g + 127) / 128;
       if (kSweep2) {
-        // Tile ti always goes to group ti & 1, so one thread owns a key's score across all query
-        // groups and can accumulate it in program order.  The queries' lse is read as broadcast
-        // float4 loads (all lanes the same address); columns past the group's rows are skipped.
-        const float* lse_g = a.lse2 + (int64_t)qrow_base + qg * kGroupRows;
-        const bool vec_ok = ((qrow_base + qg * kGroupRows) & 3) == 0;   // float4 loads need 16-byte alignment
-        const int n_full = rows_g >> 5, tail = rows_g & 31;
-        for (int ti = 0; ti < nt && ok; ++ti, ++job) {
-          if ((ti & 1) != eg) continue;
-          const int buf = job % kAccBufs;
-          ok = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), (job / kAccBufs) & 1, abort_flag, a.status));
-          if (!ok) break;
-          tc_fence_after();
-          float sum = 0.f, sum1 = 0.f;
-          for (int ch = 0; ch < n_full; ++ch) {
-            uint32_t v[32];
-            tmem_ld32(lane_addr + buf * kAccCols + ch * 32, v);
-            tmem_ld_wait();
-            if (vec_ok) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                const float4 l4 = __ldg(reinterpret_cast<const float4*>(lse_g + ch * 32 + e));
-                sum += ex2(fmaf(__uint_as_float(v[e]), c, -l4.x));
-                sum1 += ex2(fmaf(__uint_as_float(v[e + 1]), c, -l4.y));
-                sum += ex2(fmaf(__uint_as_float(v[e + 2]), c, -l4.z));
-                sum1 += ex2(fmaf(__uint_as_float(v[e + 3]), c, -l4.w));
-              }
+        // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk
+        // partials of row eg*128 + r in a fixed order, or converts the caller's value
+        if (qg > 0) epilogue_sync();                            // the previous group's values are no longer read
+        {
+          const int row = eg * 128 + r, grow = qg * kGroupRows + row;
+          float l2 = 0.f;
+          if (grow < a.rows_total) {
+            if (a.lse_in) {
+              l2 = a.lse_in[qrow_base + grow] * 1.4426950408889634f;
             } else {
+              const int rows_pad = a.n_qgroups * kGroupRows;
+              const float2* p = a.part + ((int64_t)ct.cu_chunk[b] * a.n_kv_heads + kvh) * 2 * rows_pad + grow;
+              const int64_t step = (int64_t)a.n_kv_heads * 2 * rows_pad;
+              const int nc = ct.cu_chunk[b + 1] - ct.cu_chunk[b];
+              float mx = -CUDART_INF_F;
+              for (int cc = 0; cc < nc; ++cc) {
+                mx = fmaxf(mx, p[cc * step].x);
+                mx = fmaxf(mx, p[cc * step + rows_pad].x);
+              }
+              float z = 0.f;
+              for (int cc = 0; cc < nc; ++cc) {
+                const float2 p0 = p[cc * step], p1 = p[cc * step + rows_pad];
+                z += p0.y * exp2f(p0.x - mx);
+                z += p1.y * exp2f(p1.x - mx);
+              }
+              l2 = mx + log2f(z);
+            }
+            if (a.lse_out && chunk == ct.cu_chunk[b]) a.lse_out[qrow_base + grow] = l2 * 0.6931471805599453f;
+          }
+          lse_s[row] = l2;
+        }
+        epilogue_sync();
+        // Tile ti always goes to group ti & 1, so one thread owns a key's score across both
+        // column blocks and all query groups and accumulates it in program order.
+        for (int ti = 0; ti < nt && ok; ++ti) {
+          if ((ti & 1) != eg) { job += mb; continue; }
+          float sum0 = 0.f, sum1 = 0.f;
+          for (int m = 0; m < mb && ok; ++m, ++job) {
+            const int buf = job % kAccBufs;
+            ok = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), (job / kAccBufs) & 1, abort_flag, a.status));
+            if (!ok) break;
+            tc_fence_after();
+            const int cols = min(128, rows_g - m * 128);        // query columns of this block
+            const int nch = (cols + 31) >> 5;
+            const uint32_t taddr = lane_addr + buf * kAccCols;
+            const float* lse_m = lse_s + m * 128;
+            uint32_t v[2][32];
+            tmem_ld32(taddr, v[0]);
 #pragma unroll
-              for (int e = 0; e < 32; e += 2) {
-                sum += ex2(fmaf(__uint_as_float(v[e]), c, -__ldg(lse_g + ch * 32 + e)));
-                sum1 += ex2(fmaf(__uint_as_float(v[e + 1]), c, -__ldg(lse_g + ch * 32 + e + 1)));
+            for (int ch = 0; ch < 4; ++ch) {
+              if (ch < nch) {
+                tmem_ld_wait_for(v[ch & 1]);
+                if (ch + 1 < nch) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
+                const int valid = cols - ch * 32;               // >= 32 except in the last chunk
+                if (valid >= 32) {
+#pragma unroll
+                  for (int e = 0; e < 32; e += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(lse_m + ch * 32 + e);
+                    sum0 += ex2(fmaf(__uint_as_float(v[ch & 1][e]), c, -l4.x));
+                    sum1 += ex2(fmaf(__uint_as_float(v[ch & 1][e + 1]), c, -l4.y));
+                    sum0 += ex2(fmaf(__uint_as_float(v[ch & 1][e + 2]), c, -l4.z));
+                    sum1 += ex2(fmaf(__uint_as_float(v[ch & 1][e + 3]), c, -l4.w));
+                  }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 32; ++e)
+                    if (e < valid) sum0 += ex2(fmaf(__uint_as_float(v[ch & 1][e]), c, -lse_m[ch * 32 + e]));
+                }
               }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(buf));
           }
-          if (tail) {
-            uint32_t v[32];
-            tmem_ld32(lane_addr + buf * kAccCols + n_full * 32, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (e < tail) sum += ex2(fmaf(__uint_as_float(v[e]), c, -__ldg(lse_g + n_full * 32 + e)));
-          }
-          sum += sum1;
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty(buf));
+          if (!ok) break;
           const int j = (t0 + ti) * kTileKeys + r;              // sequence-local key position
           if (j < L) {
             float* out = a.scores + (int64_t)kvh * a.score_stride + t.cu_prompt[b] + j;
+            const float sum = sum0 + sum1;
             *out = (qg == 0) ? sum : *out + sum;
           }
         }
@@ -362,19 +422,23 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
             const int i = (i_row + m * 128) % N;
             const int lim = L + i - tile_base;                  // last visible column
+            const uint32_t taddr = lane_addr + buf * kAccCols;
+            uint32_t v[2][32];
+            tmem_ld32(taddr, v[0]);
+#pragma unroll
             for (int ch = 0; ch < kTileKeys / 32; ++ch) {
-              uint32_t v[32];
-              tmem_ld32(lane_addr + buf * kAccCols + ch * 32, v);
-              tmem_ld_wait();
+              tmem_ld_wait_for(v[ch & 1]);
+              if (ch + 1 < kTileKeys / 32) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
               float x[32];
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
-                x[e] = __uint_as_float(v[e]);
+                x[e] = __uint_as_float(v[ch & 1][e]);
                 if (masked && ch * 32 + e > lim) x[e] = -CUDART_INF_F;
               }
-              float cmax = x[0];
+              float cmax = max3(x[0], x[1], x[2]);
 #pragma unroll
-              for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, x[e]);
+              for (int e = 3; e < 31; e += 2) cmax = max3(cmax, x[e], x[e + 1]);
+              cmax = fmaxf(cmax, x[31]);
               if (cmax > m_raw) {
                 z *= ex2((m_raw - cmax) * c);
                 m_raw = cmax;
@@ -413,40 +477,6 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
-}
-
-// Merge the per-chunk partials (two slots per chunk) of one pseudo query into its base-2 lse.
-__global__ void lse_merge_umma_kernel(const float2* __restrict__ part, const __grid_constant__ SeqTable t,
-                                      const __grid_constant__ ChunkTable ct, int n_q_heads, int n_kv_heads,
-                                      int n_pseudo, int rows_pad, float* __restrict__ lse2,
-                                      float* __restrict__ lse_out) {
-  const int x = blockIdx.x * blockDim.x + threadIdx.x;
-  const int per_seq = n_q_heads * n_pseudo;
-  if (x >= t.batch * per_seq) return;
-  const int b = x / per_seq, hi = x % per_seq;
-  const int rows_total = per_seq / n_kv_heads;                   // G * N
-  const int kvh = hi / rows_total, row = hi % rows_total;
-  float mx = -CUDART_INF_F;
-  for (int c = ct.cu_chunk[b]; c < ct.cu_chunk[b + 1]; ++c)
-    for (int s = 0; s < 2; ++s)
-      mx = fmaxf(mx, part[(((int64_t)c * n_kv_heads + kvh) * 2 + s) * rows_pad + row].x);
-  float z = 0.f;
-  for (int c = ct.cu_chunk[b]; c < ct.cu_chunk[b + 1]; ++c)
-    for (int s = 0; s < 2; ++s) {
-      const float2 p = part[(((int64_t)c * n_kv_heads + kvh) * 2 + s) * rows_pad + row];
-      z += p.y * exp2f(p.x - mx);
-    }
-  const float l2 = mx + log2f(z);
-  lse2[x] = l2;
-  if (lse_out) lse_out[x] = l2 * 0.6931471805599453f;
-}
-
-__global__ void lse_import_umma_kernel(const float* __restrict__ lse_in, int n, float* __restrict__ lse2,
-                                       float* __restrict__ lse_out) {
-  const int x = blockIdx.x * blockDim.x + threadIdx.x;
-  if (x >= n) return;
-  lse2[x] = lse_in[x] * 1.4426950408889634f;
-  if (lse_out) lse_out[x] = lse_in[x];
 }
 
 // ------------------------------------------------------------------------------- host side
@@ -539,7 +569,7 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
 }
 
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
-                              float2* part, float* lse2, float* scores, int64_t score_stride, float* lse_out,
+                              float2* part, float* scores, int64_t score_stride, float* lse_out,
                               int* status, cudaStream_t s, LaunchLog* log) {
   const ChunkTable& ct = plan.ct;
   UmmaArgs a;
@@ -551,10 +581,10 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   a.n_qgroups = (a.rows_total + kGroupRows - 1) / kGroupRows;
   a.has_lo = plan.has_lo;
   a.lo_row_offset = (int32_t)plan.lo_row_offset;
-  a.n_lse = t.batch * dm.n_q_heads * dm.n_pseudo;
   a.scale_log2e = dm.scale_log2e;
   a.part = part;
-  a.lse2 = lse2;
+  a.lse_in = lse_in;
+  a.lse_out = lse_out;
   a.scores = scores;
   a.score_stride = score_stride;
   a.status = status;
@@ -565,18 +595,9 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
   const dim3 grid(ct.n_chunks, dm.n_kv_heads);
-  const int n_lse = t.batch * dm.n_q_heads * dm.n_pseudo;
   if (lse_in == nullptr) {
     log->begin(kKindSweep1, s);
     k1<<<grid, kThreads, kSmemBytes, s>>>(plan.tm_k, plan.tm_q, t, ct, a);
-    log->end(s);
-    log->begin(kKindLseMerge, s);
-    lse_merge_umma_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(part, t, ct, dm.n_q_heads, dm.n_kv_heads, dm.n_pseudo,
-                                                             a.n_qgroups * kGroupRows, lse2, lse_out);
-    log->end(s);
-  } else {
-    log->begin(kKindLseMerge, s);
-    lse_import_umma_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(lse_in, n_lse, lse2, lse_out);
     log->end(s);
   }
   log->begin(kKindSweep2, s);

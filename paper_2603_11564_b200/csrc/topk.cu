@@ -1,17 +1,30 @@
 // Per-head selection of the retained tokens (Section 4.2, Eq. 5: M_retain = TopK_j S(j)).
 //
-// One CTA per (sequence, KV head).  A 4-pass, 8-bit radix select over the order-preserving
-// integer image of the fp32 scores finds the exact bit pattern of the K-th largest score
-// and how many entries equal to it still fit; an ordered compaction then writes, in
-// ascending position, every entry above the threshold plus the lowest-position ties.
+// One thread-block cluster of 8 CTAs per (sequence, KV head).  Each CTA owns a contiguous
+// slice of the head's scores and keeps their order-preserving integer images in shared
+// memory, so the scores are read from global memory once.  A 3-pass radix select (11 + 11 +
+// 10 bits, most significant first) finds the exact bit pattern of the K-th largest score and
+// how many entries equal to it still fit: per pass every CTA histograms its slice, adds its
+// non-empty bins into the cluster leader's table through distributed shared memory, and after
+// one cluster barrier every CTA scans the merged table for the digit that holds the K-th
+// entry.  An ordered compaction then writes, in ascending position, every entry above the
+// threshold plus the lowest-position ties; the CTAs learn their output offsets from each
+// other's counts, again through distributed shared memory.
 // Integer work only: the result is exact and deterministic.
+#include <cooperative_groups.h>
+
 #include "dapq_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace dapq {
 namespace {
 
 constexpr int kTopkThreads = 1024;
 constexpr int kWarps = kTopkThreads / 32;
+constexpr int kCluster = 8;                   // CTAs per (sequence, head); portable cluster size
+constexpr int kBins = 2048;                   // 11-bit digits (the last pass uses 1024 of them)
+constexpr int kMaxSliceSmem = 40960;          // keys a CTA can cache (160 KB); longer slices re-read global
 
 // Monotone map float -> uint32 (larger float <=> larger key), valid for all finite values.
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -19,113 +32,165 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(kTopkThreads)
-topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32_t* __restrict__ idx,
-                   int64_t idx_stride, const __grid_constant__ SeqTable t) {
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t s_prefix, s_remaining;
-  __shared__ uint32_t cnt_gt[kWarps], cnt_eq[kWarps];
+struct TopkSmem {
+  uint32_t merged[3][kBins];   // leader only: cluster-wide histogram of each pass
+  uint32_t hist[kBins];        // this CTA's histogram
+  uint32_t warp_sum[kWarps];
+  uint32_t cnt_gt[kWarps], cnt_eq[kWarps];
+  uint32_t cta_gt, cta_eq;     // this CTA's totals, read by the CTAs after it
+  uint32_t prefix, remaining;
+};
 
-  const int b = blockIdx.x, kvh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kTopkThreads)
+topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32_t* __restrict__ idx,
+                   int64_t idx_stride, const __grid_constant__ SeqTable t, int cache_keys) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  TopkSmem& sm = *reinterpret_cast<TopkSmem*>(smem_raw);
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TopkSmem));   // [cache_keys]
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int b = blockIdx.x / kCluster, kvh = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int L = t.prompt_len[b];
   const int K = t.cu_keep[b + 1] - t.cu_keep[b];
   const float* x = scores + (int64_t)kvh * score_stride + t.cu_prompt[b];
   int32_t* out = idx + (int64_t)kvh * idx_stride + t.cu_keep[b];
 
-  if (K >= L) {                      // keep everything
-    for (int j = tid; j < L; j += kTopkThreads) out[j] = j;
+  // slice of this CTA: [j0, j1), a multiple of 32 keys long so that warps stay converged
+  const int slice = (((L + kCluster - 1) / kCluster) + 31) & ~31;
+  const int j0 = min(L, rank * slice), j1 = min(L, j0 + slice);
+  const int n_own = j1 - j0;
+
+  if (K >= L) {                      // keep everything (uniform over the cluster: no barrier is skipped by a part of it)
+    for (int j = j0 + tid; j < j1; j += kTopkThreads) out[j] = j;
     return;
   }
 
-  if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)K; }
-  const int L_pad = (L + kTopkThreads - 1) / kTopkThreads * kTopkThreads;
+  const bool cached = slice <= cache_keys;
+  for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&sm.merged[0][0])[d] = 0u;
+  if (tid == 0) { sm.prefix = 0u; sm.remaining = (uint32_t)K; }
+  if (cached) {
+    for (int j = tid; j < n_own; j += kTopkThreads) keys[j] = order_key(x[j0 + j]);
+  }
+  cluster.sync();                    // every CTA of the cluster runs; the leader's tables are clear
 
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    const uint32_t hi_mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
-    for (int d = tid; d < 256; d += kTopkThreads) hist[d] = 0u;
+  uint32_t* leader_merged = cluster.map_shared_rank(&sm.merged[0][0], 0);
+  const int n_pad = (n_own + 31) & ~31;
+
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
+    const uint32_t hi_mask = pass == 0 ? 0u : (pass == 1 ? 0xffe00000u : 0xfffffc00u);
+    for (int d = tid; d < kBins; d += kTopkThreads) sm.hist[d] = 0u;
     __syncthreads();
-    const uint32_t prefix = s_prefix;
-    for (int j = tid; j < L_pad; j += kTopkThreads) {
+    const uint32_t prefix = sm.prefix;
+    for (int j = tid; j < n_pad; j += kTopkThreads) {
       uint32_t digit = 0xffffffffu;                       // sentinel: not a candidate
-      if (j < L) {
-        const uint32_t key = order_key(x[j]);
-        if ((key & hi_mask) == prefix) digit = (key >> shift) & 255u;
+      if (j < n_own) {
+        const uint32_t key = cached ? keys[j] : order_key(x[j0 + j]);
+        if ((key & hi_mask) == prefix) digit = (key >> shift) & digit_mask;
       }
       // one shared-memory atomic per distinct digit in the warp (scores of one head share
-      // their exponent, so most lanes hit the same bin)
+      // their exponent, so in the first pass most lanes hit the same bin)
       const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+      if (digit != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sm.hist[digit], __popc(peers));
     }
     __syncthreads();
-    if (warp == 0) {
-      // lane l owns bins 255-8l .. 248-8l (descending); find the bin holding the K-th largest
-      const uint32_t remaining = s_remaining;
-      uint32_t local[8], sum = 0u;
+    uint32_t* merged = leader_merged + pass * kBins;
+    for (int d = tid; d < kBins; d += kTopkThreads) {
+      const uint32_t c = sm.hist[d];
+      if (c) atomicAdd(merged + d, c);
+    }
+    cluster.sync();
+    // every CTA scans the merged table from the top digit down; thread t owns digits
+    // 2047-2t and 2046-2t
+    const uint32_t remaining = sm.remaining;
+    const int d_hi = kBins - 1 - 2 * tid;
+    const uint32_t v0 = merged[d_hi], v1 = merged[d_hi - 1];
+    const uint32_t mine = v0 + v1;
+    uint32_t incl = mine;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) { local[e] = hist[255 - 8 * lane - e]; sum += local[e]; }
-      uint32_t incl = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      const uint32_t hit = __ballot_sync(0xffffffffu, incl >= remaining);
-      const int owner = __ffs(hit) - 1;                   // exists: candidates >= remaining
-      if (lane == owner) {
-        uint32_t cum = incl - sum;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          if (cum + local[e] >= remaining) {
-            s_prefix = prefix | ((uint32_t)(255 - 8 * lane - e) << shift);
-            s_remaining = remaining - cum;
-            break;
-          }
-          cum += local[e];
-        }
-      }
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) sm.warp_sum[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0u;
+    for (int w = 0; w < warp; ++w) before += sm.warp_sum[w];
+    incl += before;
+    const uint32_t excl = incl - mine;
+    __syncthreads();                                       // prefix / remaining were read by everyone
+    if (excl < remaining && incl >= remaining) {           // exactly one thread
+      const bool first = excl + v0 >= remaining;
+      sm.prefix = prefix | ((uint32_t)(first ? d_hi : d_hi - 1) << shift);
+      sm.remaining = remaining - excl - (first ? 0u : v0);
     }
     __syncthreads();
   }
 
-  const uint32_t thr = s_prefix;          // key of the K-th largest score
-  const uint32_t n_ties = s_remaining;    // entries equal to it that are kept (lowest positions)
+  const uint32_t thr = sm.prefix;          // key of the K-th largest score
+  const uint32_t n_ties = sm.remaining;    // entries equal to it that are kept (lowest positions)
 
-  // ordered compaction: warp w owns the contiguous span [w * span, (w+1) * span)
-  const int span = ((L + kWarps - 1) / kWarps + 31) / 32 * 32;
-  const int j0 = warp * span, j1 = min(L, j0 + span);
+  // ordered compaction: within the CTA, warp w owns the contiguous span [w * span, (w+1) * span)
+  const int span = (((n_own + kWarps - 1) / kWarps) + 31) & ~31;
+  const int s0 = min(n_own, warp * span), s1 = min(n_own, s0 + span);
   uint32_t n_gt = 0u, n_eq = 0u;
-  for (int j = j0 + lane; j < j0 + span; j += 32) {
-    const uint32_t key = (j < j1) ? order_key(x[j]) : 0u;
-    n_gt += __popc(__ballot_sync(0xffffffffu, j < j1 && key > thr));
-    n_eq += __popc(__ballot_sync(0xffffffffu, j < j1 && key == thr));
+  for (int j = s0 + lane; j < s0 + span; j += 32) {
+    const uint32_t key = (j < s1) ? (cached ? keys[j] : order_key(x[j0 + j])) : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, j < s1 && key > thr));
+    n_eq += __popc(__ballot_sync(0xffffffffu, j < s1 && key == thr));
   }
-  if (lane == 0) { cnt_gt[warp] = n_gt; cnt_eq[warp] = n_eq; }
+  if (lane == 0) { sm.cnt_gt[warp] = n_gt; sm.cnt_eq[warp] = n_eq; }
   __syncthreads();
+  if (warp == 0) {
+    uint32_t g = sm.cnt_gt[lane], e = sm.cnt_eq[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      g += __shfl_xor_sync(0xffffffffu, g, o);
+      e += __shfl_xor_sync(0xffffffffu, e, o);
+    }
+    if (lane == 0) { sm.cta_gt = g; sm.cta_eq = e; }
+  }
+  cluster.sync();
   uint32_t gt_before = 0u, eq_before = 0u;
-  for (int w = 0; w < warp; ++w) { gt_before += cnt_gt[w]; eq_before += cnt_eq[w]; }
+  for (int r = 0; r < rank; ++r) {
+    gt_before += *cluster.map_shared_rank(&sm.cta_gt, r);
+    eq_before += *cluster.map_shared_rank(&sm.cta_eq, r);
+  }
+  for (int w = 0; w < warp; ++w) { gt_before += sm.cnt_gt[w]; eq_before += sm.cnt_eq[w]; }
   uint32_t pos = gt_before + min(eq_before, n_ties);
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (int j = j0 + lane; j < j0 + span; j += 32) {
-    const uint32_t key = (j < j1) ? order_key(x[j]) : 0u;
-    const bool gt = j < j1 && key > thr;
-    const bool eq = j < j1 && key == thr;
+  for (int j = s0 + lane; j < s0 + span; j += 32) {
+    const uint32_t key = (j < s1) ? (cached ? keys[j] : order_key(x[j0 + j])) : 0u;
+    const bool gt = j < s1 && key > thr;
+    const bool eq = j < s1 && key == thr;
     const uint32_t eq_bal = __ballot_sync(0xffffffffu, eq);
     const bool take = gt || (eq && eq_before + __popc(eq_bal & lt_mask) < n_ties);
     const uint32_t take_bal = __ballot_sync(0xffffffffu, take);
-    if (take) out[pos + __popc(take_bal & lt_mask)] = j;
+    if (take) out[pos + __popc(take_bal & lt_mask)] = j0 + j;
     pos += __popc(take_bal);
     eq_before += __popc(eq_bal);
   }
+  cluster.sync();                    // no CTA exits while another may still read its counts
 }
 
 }  // namespace
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log) {
+  int max_len = 1;
+  for (int b = 0; b < t.batch; ++b) max_len = t.prompt_len[b] > max_len ? t.prompt_len[b] : max_len;
+  const int slice = (((max_len + kCluster - 1) / kCluster) + 31) & ~31;
+  const int cache_keys = slice <= kMaxSliceSmem ? slice : 0;          // 0: every pass re-reads global memory
+  const size_t smem = sizeof(TopkSmem) + (size_t)cache_keys * sizeof(uint32_t);
+  cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(sizeof(TopkSmem) + (size_t)kMaxSliceSmem * sizeof(uint32_t)));
+  if (e != cudaSuccess) return e;
   log->begin(kKindTopk, s);
-  topk_select_kernel<<<dim3(t.batch, n_kv_heads), kTopkThreads, 0, s>>>(scores, score_stride, idx,
-                                                                        idx_stride, t);
+  topk_select_kernel<<<dim3(t.batch * kCluster, n_kv_heads), kTopkThreads, smem, s>>>(scores, score_stride, idx,
+                                                                                      idx_stride, t, cache_keys);
   log->end(s);
   return cudaGetLastError();
 }

@@ -171,9 +171,12 @@ def test_score_strided_view_and_custom_scale(dq):
 
 
 # -------------------------------------------------------------------------- dapq_topk_select
-def test_topk_exact_with_ties(dq):
+@pytest.mark.parametrize("lens,keep", [
+    ((1, 33, 4096, 5000, 131072, 77), (1, 33, 1, 4999, 3932, 200)),
+    ((400000, 9), (12345, 3)),       # slices too long for the shared-memory key cache
+])
+def test_topk_exact_with_ties(dq, lens, keep):
     rng = np.random.default_rng(5)
-    lens, keep = (1, 33, 4096, 5000, 131072, 77), (1, 33, 1, 4999, 3932, 200)
     w = _small(lens=lens, keep=keep, n_q_heads=3, n_kv_heads=3, n_pseudo=4, n_needles=0, outlier_channels=0)
     T = w.total_prompt
     s = rng.random((3, T)).astype(np.float32)
