@@ -98,6 +98,7 @@ cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const Ca
 struct UmmaPlan {
   CUtensorMap tm_k, tm_q;
   ChunkTable ct;
+  const void* q_hi;
   int32_t has_lo;
   int64_t lo_row_offset;
 };
