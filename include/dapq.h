@@ -187,6 +187,34 @@ DAPQ_API dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, cons
                             const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
                             int32_t* idx_out_host, void* stream);
 
+/* The paper has no counterpart to this entry point; it exists for callers that may not
+ * allocate device memory at the point where they need scores: engines whose own allocator owns
+ * the whole device, plug-ins running after a "no more driver allocations" point, code between a
+ * memory-pool snapshot and its restore.  dapq_create allocates a workspace, so such callers
+ * cannot build a context; this call needs none and calls no cudaMalloc / cudaFree or any
+ * allocating library routine.
+ *
+ * It computes what dapq_score computes (Eq. 4 scores per KV head, fp32 arithmetic on the CUDA
+ * cores, both sweeps) from shape fields only: n_q_heads, n_kv_heads, head_dim, n_pseudo, dtype
+ * and softmax_scale of `shape` are read, the rest is ignored.  q_rot (device, already rotated,
+ * element type shape->dtype), cache->k (device) and scores (device, [H_kv, T]) are the caller's;
+ * cache->v is not read.
+ *
+ * The scratch of the two sweeps lives in one fixed array of DAPQ_STATIC_SCRATCH_BYTES inside
+ * the library image, which every GPU that loads the library holds until the process exits.  A
+ * call needs  sum_b (ceil(L_b / 512) + 1) * H_q * N * 8  +  B * H_q * N * 4  bytes of it (e.g.
+ * 64k prompt tokens at H_q = 32, N = 64); a larger call returns DAPQ_ERR_WORKSPACE and launches
+ * nothing.  All calls on a device share the array: calls whose kernels can overlap on the GPU
+ * (different streams, no dependency) race on it and must be ordered by the caller.  Nothing in
+ * it needs clearing between calls.  The first call on each device resolves the array's device
+ * address (a one-time, per-device set-up with that device current); make that first call
+ * outside any stream capture.
+ * err_out (nullable, host): receives a NUL-terminated reason when the status is not DAPQ_OK. */
+enum { DAPQ_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024 };
+DAPQ_API dapq_status dapq_score_static(const dapq_shape* shape, int device, const void* q_rot,
+                              const dapq_cache_view* cache, float* scores, void* stream,
+                              char* err_out, size_t err_len);
+
 #ifdef __cplusplus
 }
 #endif

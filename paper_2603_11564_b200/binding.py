@@ -27,7 +27,7 @@ _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORT
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
            "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
-           "dapq_compact_kv", "dapq_evict", "dapq_evict_host")
+           "dapq_compact_kv", "dapq_evict", "dapq_evict_host", "dapq_score_static")
 
 
 class DapqError(RuntimeError):
@@ -90,6 +90,9 @@ def load_library() -> C.CDLL:
     lib.dapq_evict.restype = C.c_int
     lib.dapq_evict_host.argtypes = [vp, vp, C.POINTER(dapq_cache_view), i32p, vp, vp, vp, vp]
     lib.dapq_evict_host.restype = C.c_int
+    lib.dapq_score_static.argtypes = [C.POINTER(dapq_shape), C.c_int, vp, C.POINTER(dapq_cache_view), f32p, vp,
+                                      C.c_char_p, C.c_size_t]
+    lib.dapq_score_static.restype = C.c_int
     _lib = lib
     return lib
 
@@ -232,3 +235,23 @@ def dapq_evict_host(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, 
     kk, kk_p = _i32(k_keep)
     _check(ctx, load_library().dapq_evict_host(ctx, q_pre.data_ptr(), C.byref(view), kk_p, k_out.data_ptr(),
                                                v_out.data_ptr(), _ptr(idx_out), _stream(stream)))
+
+
+DAPQ_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
+
+
+def dapq_score_static(n_q_heads: int, n_kv_heads: int, n_pseudo: int, dtype: int, q_rot: torch.Tensor,
+                      k: torch.Tensor, cu_rows, prompt_len, scores: torch.Tensor, softmax_scale: float = 0.0,
+                      head_dim: int = 128, device: int = 0, stream=None) -> None:
+    """dapq_score for callers that may not allocate device memory (no context, no workspace:
+    the scratch is a fixed array inside the library).  Raises DapqError(DAPQ_ERR_WORKSPACE)
+    when the call needs more than DAPQ_STATIC_SCRATCH_BYTES of scratch."""
+    sh = dapq_shape(n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim, n_pseudo=n_pseudo,
+                    max_batch=len(prompt_len), dtype=dtype, max_total_rows=int(cu_rows[-1]), rope_base=1.0,
+                    softmax_scale=softmax_scale)
+    view = _view(k, None, cu_rows, prompt_len)
+    err = C.create_string_buffer(512)
+    st = load_library().dapq_score_static(C.byref(sh), device, q_rot.data_ptr(), C.byref(view), scores.data_ptr(),
+                                          _stream(stream), err, len(err))
+    if st != DAPQ_OK:
+        raise DapqError(st, err.value.decode())
