@@ -27,7 +27,7 @@ struct SeqTable {
 
 // How the score sweeps cut the sequences into work chunks (one CTA per chunk and KV head).
 //   CUDA-core path:   chunks of kChunkKeys prompt keys, then one chunk with the N synthetic rows;
-//   tensor-core path: chunks of chunk_tiles 128-row tiles over the rows [0, L_b + N).
+//   tensor-core path: chunks of chunk_tiles whole K tiles (the tile size is the sweep's).
 struct ChunkTable {
   int32_t chunk_tiles;
   int32_t n_chunks;
@@ -96,9 +96,8 @@ cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const Ca
 // CUDA-core path).  q_hi: [B*H_q*N, d] bf16; with has_lo the low-order parts follow
 // lo_row_offset rows later in the same allocation.
 struct UmmaPlan {
-  CUtensorMap tm_k, tm_q;
-  ChunkTable ct;
-  const void* q_hi;
+  CUtensorMap tm_k1, tm_k2, tm_q;   // K for sweep 1 / sweep 2 (different boxes), the query operand
+  ChunkTable ct1, ct2;              // work cut of sweep 1 (192-key tiles over L_b + N) / sweep 2 (128-key tiles over L_b)
   int32_t has_lo;
   int64_t lo_row_offset;
 };

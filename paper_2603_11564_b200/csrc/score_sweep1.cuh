@@ -1,0 +1,173 @@
+// Sweep 1 of the tensor-core scorer: per pseudo query, the running maximum and the sum of
+// exponentials of its logits over the CTA's chunk of keys (Appendix C, Step 1: s_j = q k_j /
+// sqrt(d_k); the softmax normaliser of Section 4.2, Eq. 4 is built from these partials).
+//
+//   D[query, key] = Q_blk K_tile^T, queries on tensor-memory lanes, 192 keys per tile.
+// A job is one [128 queries x 192 keys] accumulator; the two query blocks of a group own one
+// accumulator each, so the MMAs of one block run while the other block's accumulator is read.
+// Both epilogue groups work on every job, 96 key columns each: thread (group g, row r) keeps
+// the statistics of query row r over the columns of its group, which become slot g of the
+// row's per-chunk partials.
+#pragma once
+#include "score_umma_common.cuh"
+
+namespace dapq {
+namespace umma {
+
+// Running max / sum of exp over one 32-column piece of an accumulator row.
+// lim: last visible column of the piece's tile for this thread's pseudo query (masked tiles).
+template <bool kMasked>
+__device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int lim, float c, float& m_raw, float& z) {
+  float x[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    x[e] = __uint_as_float(v[e]);
+    if (kMasked && col0 + e > lim) x[e] = -CUDART_INF_F;
+  }
+  float cmax = max3(x[0], x[1], x[2]);
+#pragma unroll
+  for (int e = 3; e < 31; e += 2) cmax = max3(cmax, x[e], x[e + 1]);
+  cmax = fmaxf(cmax, x[31]);
+  if (cmax > m_raw) {
+    z *= ex2((m_raw - cmax) * c);
+    m_raw = cmax;
+  }
+  if (!kMasked || m_raw > -CUDART_INF_F) {
+    const float neg = -m_raw * c;
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+      s0 += ex2(fmaf(x[e], c, neg));
+      s1 += ex2(fmaf(x[e + 1], c, neg));
+    }
+    z += s0 + s1;
+  }
+}
+
+// This group's 96 columns of one accumulator, in three pieces with the next piece's load in flight.
+__device__ __forceinline__ void row_stats_job(uint32_t taddr, int col0, bool masked, int lim, float c, float& m_raw,
+                                              float& z) {
+  uint32_t v[2][32];
+  tmem_ld32(taddr, v[0]);
+#pragma unroll
+  for (int ch = 0; ch < 3; ++ch) {
+    tmem_ld_wait_for(v[ch & 1]);
+    if (ch + 1 < 3) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
+    if (masked) row_stats_piece<true>(v[ch & 1], col0 + ch * 32, lim, c, m_raw, z);
+    else row_stats_piece<false>(v[ch & 1], col0 + ch * 32, lim, c, m_raw, z);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                    const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct, const UmmaArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x, kvh = blockIdx.y;
+  const Work w = cta_work(t, ct, a, kTile1, true);
+  const int nt = w.nt, L = w.L, N = a.n_pseudo;
+  if (nt <= 0) return;
+  const Bars bars{sbase + Smem::bars};
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages1);
+
+  if (warp == 0) {
+    if (lane == 0)
+      tma_producer<kTile1, kStages1, kStageBytes1, kHalfBytes1>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
+  } else if (warp == 1) {
+    // ============================================================================= MMA issuer
+    if (lane == 0) {
+      int li = 0;
+      uint32_t use0 = 0u, use1 = 0u;                            // jobs issued into each accumulator
+      bool ok = true;
+      const uint32_t idesc = umma_idesc(128, kTile1);
+      const uint64_t qd_hi = umma_desc(sbase + Smem::q_hi), qd_lo = umma_desc(sbase + Smem::q_lo);
+      for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+        const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+        const int mb = (rows_g + 127) / 128;
+        ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
+        for (int ti = 0; ti < nt && ok; ++ti, ++li) {
+          const int s = li % kStages1;
+          ok = mbar_wait(bars.k_full(s), (li / kStages1) & 1, abort_flag, a.status);
+          if (!ok) break;
+          const uint64_t kd = umma_desc(sbase + Smem::k + s * kStageBytes1);
+          for (int m = 0; m < mb && ok; ++m) {
+            // two blocks: block m -> accumulator m; one block: tiles alternate between the two
+            const int buf = (mb == 2) ? m : (ti & 1);
+            const uint32_t used = buf ? use1 : use0;
+            if (used) ok = mbar_wait(bars.acc_empty(buf), (used - 1) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d = tmem_base + buf * kTile1;
+            const uint64_t qh = desc_advance(qd_hi, m * 128 * 128), ql = desc_advance(qd_lo, m * 128 * 128);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const int half = ks >> 2, kk = ks & 3;
+              umma_ss(d, desc_advance(qh, half * kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
+                      idesc, ks ? 1u : 0u);
+            }
+            if (a.has_lo) {
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const int half = ks >> 2, kk = ks & 3;
+                umma_ss(d, desc_advance(ql, half * kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
+                        idesc, 1u);
+              }
+            }
+            tc_commit(bars.acc_full(buf));
+            if (buf) ++use1; else ++use0;
+          }
+          tc_commit(bars.k_empty(s));                           // the K stage is free once these MMAs retire
+        }
+        tc_commit(bars.q_empty());
+      }
+    }
+  } else {
+    // ============================================================================== epilogue
+    const int eg = (warp - 2) >> 2;                             // epilogue group 0 / 1: key columns 96 eg .. 96 eg + 95
+    const int quad = warp & 3;                                  // TMEM lane quadrant of this warp
+    const int r = quad * 32 + lane;                             // accumulator row of this thread
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const float c = a.scale_log2e;
+    const int col0 = eg * (kTile1 / 2);
+    uint32_t use0 = 0u, use1 = 0u;                              // jobs taken from each accumulator
+    bool ok = true;
+    for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+      const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+      const int mb = (rows_g + 127) / 128;
+      // running max (raw dot product) and sum of this thread's row of block 0 / block 1
+      float m_raw0 = -CUDART_INF_F, z0 = 0.f, m_raw1 = -CUDART_INF_F, z1 = 0.f;
+      const int i_q0 = (qg * kGroupRows + r) % N, i_q1 = (qg * kGroupRows + 128 + r) % N;   // pseudo-query indices
+      for (int ti = 0; ti < nt && ok; ++ti) {
+        const int tile_base = (w.t0 + ti) * kTile1;
+        const bool masked = tile_base + kTile1 > L;             // holds synthetic (or foreign) rows
+        for (int m = 0; m < mb && ok; ++m) {
+          const int buf = (mb == 2) ? m : (ti & 1);
+          const uint32_t used = buf ? use1 : use0;
+          ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), used & 1, abort_flag, a.status));
+          if (!ok) break;
+          if (buf) ++use1; else ++use0;
+          tc_fence_after();
+          const uint32_t taddr = lane_addr + buf * kTile1 + col0;
+          // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
+          if (m == 0) row_stats_job(taddr, col0, masked, L + i_q0 - tile_base, c, m_raw0, z0);
+          else row_stats_job(taddr, col0, masked, L + i_q1 - tile_base, c, m_raw1, z1);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+        }
+      }
+      // partials: slot eg of this thread's rows
+      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * 2 + eg) * (a.n_qgroups * kGroupRows) +
+                      qg * kGroupRows;
+      if (qg * kGroupRows + r < a.rows_total) pbase[r] = make_float2(m_raw0 * c, z0);
+      if (mb == 2 && qg * kGroupRows + 128 + r < a.rows_total) pbase[128 + r] = make_float2(m_raw1 * c, z1);
+    }
+  }
+  cta_epilogue(tmem_base);
+}
+
+}  // namespace umma
+}  // namespace dapq

@@ -1,0 +1,182 @@
+// Sweep 2 of the tensor-core scorer (Section 4.2, Eq. 4): S(j) = sum_i exp(s_ij - lse_i),
+// summed over the N pseudo queries and the G query heads of the KV head's group.
+//
+//   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
+// A job is one [128 keys x 256 queries] accumulator (two fit).  Both epilogue groups work on
+// every job, half of the query columns each; group 1 hands its partial sum to group 0 through
+// a consumed column of the same accumulator, and group 0's thread (lane = key) stores the
+// key's score: one coalesced fp32 per lane.  Before the first job the epilogue threads merge
+// the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the resident query rows.
+#pragma once
+#include "score_umma_common.cuh"
+
+namespace dapq {
+namespace umma {
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                    const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
+                    const __grid_constant__ ChunkTable ct1, const UmmaArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x, kvh = blockIdx.y;
+  const Work w = cta_work(t, ct, a, kTile2, false);
+  const int nt = w.nt, L = w.L, b = w.b;
+  if (nt <= 0) return;
+  const Bars bars{sbase + Smem::bars};
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
+  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] base-2 lse of the resident query group
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages2);
+
+  if (warp == 0) {
+    if (lane == 0)
+      tma_producer<kTile2, kStages2, kStageBytes2, kHalfBytes2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
+  } else if (warp == 1) {
+    // ============================================================================= MMA issuer
+    if (lane == 0) {
+      int job = 0;                                              // = K tiles consumed: one job per tile
+      bool ok = true;
+      const uint64_t qd_hi = umma_desc(sbase + Smem::q_hi), qd_lo = umma_desc(sbase + Smem::q_lo);
+      for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+        const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+        const uint32_t idesc = umma_idesc(128, (rows_g + 15) & ~15);   // only the query columns that exist
+        ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
+        for (int ti = 0; ti < nt && ok; ++ti, ++job) {
+          const int s = job % kStages2, buf = job & 1;
+          ok = mbar_wait(bars.k_full(s), (job / kStages2) & 1, abort_flag, a.status);
+          if (ok && job >= 2) ok = mbar_wait(bars.acc_empty(buf), ((job >> 1) - 1) & 1, abort_flag, a.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t kd = umma_desc(sbase + Smem::k + s * kStageBytes2);
+          const uint32_t d = tmem_base + buf * 256;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const int half = ks >> 2, kk = ks & 3;
+            umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * kHalfBytesQ + kk * 32),
+                    idesc, ks ? 1u : 0u);
+          }
+          if (a.has_lo) {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const int half = ks >> 2, kk = ks & 3;
+              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_lo, half * kHalfBytesQ + kk * 32),
+                      idesc, 1u);
+            }
+          }
+          tc_commit(bars.acc_full(buf));
+          tc_commit(bars.k_empty(s));                           // the K stage is free once these MMAs retire
+        }
+        tc_commit(bars.q_empty());
+      }
+    }
+  } else {
+    // ============================================================================== epilogue
+    const int eg = (warp - 2) >> 2;                             // epilogue group 0 / 1
+    const int quad = warp & 3;                                  // TMEM lane quadrant of this warp
+    const int r = quad * 32 + lane;                             // accumulator row of this thread
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const float c = a.scale_log2e;
+    int job = 0;
+    bool ok = true;
+    // (an aborting group still walks every query group: the other group waits for it at the barriers)
+    for (int qg = 0; qg < a.n_qgroups; ++qg) {
+      const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+      // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk
+      // partials of row eg*128 + r in a fixed order, or converts the caller's value
+      if (qg > 0) epilogue_sync();                              // the previous group's values are no longer read
+      {
+        const int row = eg * 128 + r, grow = qg * kGroupRows + row;
+        float l2 = 0.f;
+        if (grow < a.rows_total) {
+          if (a.lse_in) {
+            l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
+          } else {
+            const int rows_pad = a.n_qgroups * kGroupRows;
+            const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * 2 * rows_pad + grow;
+            const int64_t step = (int64_t)a.n_kv_heads * 2 * rows_pad;
+            const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
+            float mx = -CUDART_INF_F;
+            for (int cc = 0; cc < nc; ++cc) {
+              mx = fmaxf(mx, p[cc * step].x);
+              mx = fmaxf(mx, p[cc * step + rows_pad].x);
+            }
+            float z = 0.f;
+            for (int cc = 0; cc < nc; ++cc) {
+              const float2 p0 = p[cc * step], p1 = p[cc * step + rows_pad];
+              z += p0.y * exp2f(p0.x - mx);
+              z += p1.y * exp2f(p1.x - mx);
+            }
+            l2 = mx + log2f(z);
+          }
+          if (a.lse_out && chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
+        }
+        lse_s[row] = l2;
+      }
+      epilogue_sync();
+      // 32-column pieces of a job: group 0 takes the first h, group 1 the rest
+      const int nch = (rows_g + 31) >> 5, h = (nch + 1) >> 1;
+      const int p0 = eg ? h : 0, np = eg ? nch - h : h;
+      for (int ti = 0; ti < nt && ok; ++ti, ++job) {
+        const int buf = job & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), (job >> 1) & 1, abort_flag, a.status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = lane_addr + buf * 256;
+        float sum0 = 0.f, sum1 = 0.f;
+        uint32_t v[2][32];
+        if (np > 0) tmem_ld32(taddr + p0 * 32, v[0]);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (k < np) {
+            tmem_ld_wait_for(v[k & 1]);
+            if (k + 1 < np) tmem_ld32(taddr + (p0 + k + 1) * 32, v[(k + 1) & 1]);
+            const int ch = p0 + k;
+            const int valid = rows_g - ch * 32;                 // >= 32 except in the last piece
+            if (valid >= 32) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
+                sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, -l4.x));
+                sum1 += ex2(fmaf(__uint_as_float(v[k & 1][e + 1]), c, -l4.y));
+                sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e + 2]), c, -l4.z));
+                sum1 += ex2(fmaf(__uint_as_float(v[k & 1][e + 3]), c, -l4.w));
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (e < valid) sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, -lse_s[ch * 32 + e]));
+            }
+          }
+        }
+        float sum = sum0 + sum1;
+        const uint32_t xcol = taddr + h * 32;                   // a column group 1 has consumed (or nobody reads)
+        if (eg == 1) {
+          tmem_st1(xcol, __float_as_uint(sum));
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(bars.half_done(buf)); mbar_arrive(bars.acc_empty(buf)); }
+        } else {
+          ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job >> 1) & 1, abort_flag, a.status));
+          if (!ok) break;
+          tc_fence_after();
+          sum += __uint_as_float(tmem_ld1(xcol));
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+          const int j = (w.t0 + ti) * kTile2 + r;               // sequence-local key position
+          if (j < L) {
+            float* out = a.scores + (int64_t)kvh * a.score_stride + t.cu_prompt[b] + j;
+            *out = (qg == 0) ? sum : *out + sum;
+          }
+        }
+      }
+    }
+  }
+  cta_epilogue(tmem_base);
+}
+
+}  // namespace umma
+}  // namespace dapq

@@ -1,0 +1,162 @@
+// Definitions shared by the two sweeps of the tensor-core scorer (see score_umma.cu).
+#pragma once
+#include "umma_ptx.cuh"
+
+namespace dapq {
+namespace umma {
+
+using namespace ptx;
+
+constexpr int kTile1 = 192;                    // keys per K tile of sweep 1 (= UMMA N there)
+constexpr int kTile2 = 128;                    // keys per K tile of sweep 2 (= UMMA M there)
+constexpr int kGroupRows = 256;                // query rows resident per group (2 blocks of 128)
+constexpr int kHalfBytesQ = kGroupRows * 128;  // one 64-channel half of a query group (32 KB)
+constexpr int kQBytes = 2 * kHalfBytesQ;       // 64 KB per precision part (hi / lo)
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 512;
+
+// Shared memory of both sweeps (offsets from the 1024-aligned base): the query group as a
+// bf16 pair, a K ring of 96 KB (2 x 192 keys in sweep 1, 3 x 128 keys in sweep 2), barriers,
+// and (sweep 2) the group's log-sum-exp.
+constexpr int kStages1 = 2, kStageBytes1 = kTile1 * 256, kHalfBytes1 = kTile1 * 128;
+constexpr int kStages2 = 3, kStageBytes2 = kTile2 * 256, kHalfBytes2 = kTile2 * 128;
+struct Smem {
+  static constexpr int q_hi = 0;
+  static constexpr int q_lo = q_hi + kQBytes;
+  static constexpr int k = q_lo + kQBytes;
+  static constexpr int bars = k + 96 * 1024;
+  // barriers (16 x 8 B): k_full[3], k_empty[3], acc_full[2], acc_empty[2], q_full, q_empty, half_done[2]
+  static constexpr int lse = bars + 16 * 8;          // [256] floats
+  static constexpr int tmem_ptr = lse + kGroupRows * 4;
+  static constexpr int abort_flag = tmem_ptr + 4;
+  static constexpr int total = abort_flag + 4;
+};
+static_assert(kStages1 * kStageBytes1 == 96 * 1024 && kStages2 * kStageBytes2 == 96 * 1024, "K ring is 96 KB");
+constexpr int kSmemBytes = Smem::total + 1024;   // slack for the manual 1024-byte alignment
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
+
+struct UmmaArgs {
+  int32_t n_pseudo, group, n_q_heads, n_kv_heads;
+  int32_t rows_total;        // G * N
+  int32_t n_qgroups;         // ceil(rows_total / 256)
+  int32_t has_lo;            // the query operand carries a low-order bf16 part
+  int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
+  float scale_log2e;
+  float2* part;              // [n_chunks1, H_kv, 2, n_qgroups * 256] (running max, sum) in base 2
+  const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
+  float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
+  float* scores;
+  int64_t score_stride;
+  int* status;
+};
+
+// This CTA's work: sequence, tile range, first cache row and first query row.
+struct Work {
+  int b, L, nt, t0, row_base, qrow_base;
+};
+// n_keys(b): keys of sequence b that the sweep covers (L_b + N in sweep 1, L_b in sweep 2).
+__device__ __forceinline__ Work cta_work(const SeqTable& t, const ChunkTable& ct, const UmmaArgs& a, int tile_keys,
+                                         bool with_synthetic) {
+  Work w;
+  const int chunk = blockIdx.x, kvh = blockIdx.y;
+  w.b = find_segment(ct.cu_chunk, t.batch, chunk);
+  w.L = t.prompt_len[w.b];
+  const int n_keys = w.L + (with_synthetic ? a.n_pseudo : 0);
+  const int n_tiles = (n_keys + tile_keys - 1) / tile_keys;
+  w.t0 = (chunk - ct.cu_chunk[w.b]) * ct.chunk_tiles;
+  w.nt = min(n_tiles, w.t0 + ct.chunk_tiles) - w.t0;
+  w.row_base = t.cu_rows[w.b];                                          // first cache row of the sequence
+  w.qrow_base = (w.b * a.n_q_heads + kvh * a.group) * a.n_pseudo;       // first query row of this KV head
+  return w;
+}
+
+// Barrier addresses of a CTA.
+struct Bars {
+  uint32_t base;
+  __device__ __forceinline__ uint32_t k_full(int s) const { return base + 8u * s; }
+  __device__ __forceinline__ uint32_t k_empty(int s) const { return base + 8u * (3 + s); }
+  __device__ __forceinline__ uint32_t acc_full(int i) const { return base + 8u * (6 + i); }
+  __device__ __forceinline__ uint32_t acc_empty(int i) const { return base + 8u * (8 + i); }
+  __device__ __forceinline__ uint32_t q_full() const { return base + 8u * 10; }
+  __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * 11; }
+  __device__ __forceinline__ uint32_t half_done(int i) const { return base + 8u * (12 + i); }
+};
+
+// Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync.
+// Returns the tensor-memory base address.
+__device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, int n_stages) {
+  const int warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) { mbar_init(bars.k_full(s), 1); mbar_init(bars.k_empty(s), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars.acc_full(i), 1);
+      mbar_init(bars.acc_empty(i), 8);      // all 8 epilogue warps read every accumulator
+      mbar_init(bars.half_done(i), 4);
+    }
+    mbar_init(bars.q_full(), 1);
+    mbar_init(bars.q_empty(), 1);
+    *reinterpret_cast<volatile int*>(smem + Smem::abort_flag) = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {                                              // tensor memory: all 512 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(sbase + Smem::tmem_ptr), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  return *reinterpret_cast<volatile uint32_t*>(smem + Smem::tmem_ptr);
+}
+
+__device__ __forceinline__ void cta_epilogue(uint32_t tmem_base) {
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// TMA producer loop shared by both sweeps: per query group the query blocks (hi, lo), then the
+// CTA's K tiles through the ring.  kTile / kStages / kHalf are the sweep's tile geometry.
+template <int kTile, int kStages, int kStage, int kHalf>
+__device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w,
+                                             const UmmaArgs& a, uint32_t sbase, const Bars& bars, int kvh,
+                                             volatile int* abort_flag) {
+  int li = 0;                                               // K tiles loaded so far
+  bool ok = true;
+  for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+    const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+    const int mb = (rows_g + 127) / 128;
+    if (qg > 0) ok = mbar_wait(bars.q_empty(), (qg - 1) & 1, abort_flag, a.status);
+    if (!ok) break;
+    const int parts = a.has_lo ? 2 : 1;
+    mbar_expect_tx(bars.q_full(), (uint32_t)(parts * mb * 2 * 128 * 128));
+    for (int part = 0; part < parts; ++part)
+      for (int half = 0; half < 2; ++half)
+        for (int m = 0; m < mb; ++m)
+          tma_load_2d(sbase + (part ? Smem::q_lo : Smem::q_hi) + half * kHalfBytesQ + m * 128 * 128, tm_q, bars.q_full(),
+                      half * 64, part * a.lo_row_offset + w.qrow_base + qg * kGroupRows + m * 128);
+    for (int ti = 0; ti < w.nt; ++ti, ++li) {
+      const int s = li % kStages;
+      if (li >= kStages) ok = mbar_wait(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status);
+      if (!ok) break;
+      mbar_expect_tx(bars.k_full(s), kStage);
+      const int row = w.row_base + (w.t0 + ti) * kTile;
+      tma_load_3d(sbase + Smem::k + s * kStage, tm_k, bars.k_full(s), 0, row, kvh);
+      tma_load_3d(sbase + Smem::k + s * kStage + kHalf, tm_k, bars.k_full(s), 64, row, kvh);
+    }
+  }
+  if (!ok) {
+    // aborting: let the copies already issued land before the CTA returns
+    for (int back = 1; back <= kStages && back <= li; ++back) {
+      const int l2 = li - back;
+      const long long start = clock64();
+      while (!mbar_try(bars.k_full(l2 % kStages), (l2 / kStages) & 1) && clock64() - start < kWaitLimit) {}
+    }
+  }
+}
+
+}  // namespace umma
+}  // namespace dapq
