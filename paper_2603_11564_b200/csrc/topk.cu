@@ -4,12 +4,14 @@
 // slice of the head's scores and keeps their order-preserving integer images in shared
 // memory, so the scores are read from global memory once.  A 3-pass radix select (11 + 11 +
 // 10 bits, most significant first) finds the exact bit pattern of the K-th largest score and
-// how many entries equal to it still fit: per pass every CTA histograms its slice, adds its
-// non-empty bins into the cluster leader's table through distributed shared memory, and after
-// one cluster barrier every CTA scans the merged table for the digit that holds the K-th
-// entry.  An ordered compaction then writes, in ascending position, every entry above the
-// threshold plus the lowest-position ties; the CTAs learn their output offsets from each
-// other's counts, again through distributed shared memory.
+// how many entries equal to it still fit: per pass every CTA histograms its slice with plain
+// shared-memory atomics, adds its non-empty bins into the table of EVERY CTA of the cluster
+// through distributed shared memory (remote adds need no reply), and after one cluster barrier
+// scans its own copy of the merged table for the digit that holds the K-th entry.  After the
+// first pass a CTA keeps only its candidates (the keys of the selected bin) in a short list, so
+// the later passes touch few keys.  An ordered compaction then writes, in ascending position,
+// every entry above the threshold plus the lowest-position ties; the CTAs push their counts to
+// each other the same way, so no CTA reads remote memory and none has to outlive another.
 // Integer work only: the result is exact and deterministic.
 #include <cooperative_groups.h>
 
@@ -24,7 +26,8 @@ constexpr int kTopkThreads = 1024;
 constexpr int kWarps = kTopkThreads / 32;
 constexpr int kCluster = 8;                   // CTAs per (sequence, head); portable cluster size
 constexpr int kBins = 2048;                   // 11-bit digits (the last pass uses 1024 of them)
-constexpr int kMaxSliceSmem = 40960;          // keys a CTA can cache (160 KB); longer slices re-read global
+constexpr int kMaxSliceSmem = 36864;          // keys a CTA can cache (144 KB); longer slices re-read global
+constexpr int kMaxCand = 4096;                // candidate keys a CTA lists after the first pass
 
 // Monotone map float -> uint32 (larger float <=> larger key), valid for all finite values.
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -33,12 +36,13 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 struct TopkSmem {
-  uint32_t merged[3][kBins];   // leader only: cluster-wide histogram of each pass
-  uint32_t hist[kBins];        // this CTA's histogram
+  uint32_t merged[3][kBins];   // cluster-wide histogram of each pass (every CTA holds a copy)
+  uint32_t hist[kBins];        // this CTA's histogram (all zero between passes)
+  uint32_t cand[kMaxCand];     // this CTA's keys that share the first pass's digit
   uint32_t warp_sum[kWarps];
   uint32_t cnt_gt[kWarps], cnt_eq[kWarps];
-  uint32_t cta_gt, cta_eq;     // this CTA's totals, read by the CTAs after it
-  uint32_t prefix, remaining;
+  uint32_t peer_gt[kCluster], peer_eq[kCluster];   // totals of every CTA of the cluster, pushed by their owners
+  uint32_t prefix, remaining, n_cand;
 };
 
 __global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kTopkThreads)
@@ -69,45 +73,47 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
 
   const bool cached = slice <= cache_keys;
   for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&sm.merged[0][0])[d] = 0u;
-  if (tid == 0) { sm.prefix = 0u; sm.remaining = (uint32_t)K; }
+  for (int d = tid; d < kBins; d += kTopkThreads) sm.hist[d] = 0u;
+  if (tid == 0) { sm.prefix = 0u; sm.remaining = (uint32_t)K; sm.n_cand = 0u; }
   if (cached) {
     for (int j = tid; j < n_own; j += kTopkThreads) keys[j] = order_key(x[j0 + j]);
   }
-  cluster.sync();                    // every CTA of the cluster runs; the leader's tables are clear
+  cluster.sync();                    // every CTA of the cluster runs and has cleared its tables
 
-  uint32_t* leader_merged = cluster.map_shared_rank(&sm.merged[0][0], 0);
-  const int n_pad = (n_own + 31) & ~31;
+  uint32_t* peer_merged[kCluster];
+#pragma unroll
+  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&sm.merged[0][0], p);
+  bool listed = false;               // the later passes read the candidate list instead of the slice
 
   for (int pass = 0; pass < 3; ++pass) {
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
     const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
     const uint32_t hi_mask = pass == 0 ? 0u : (pass == 1 ? 0xffe00000u : 0xfffffc00u);
-    for (int d = tid; d < kBins; d += kTopkThreads) sm.hist[d] = 0u;
-    __syncthreads();
     const uint32_t prefix = sm.prefix;
-    for (int j = tid; j < n_pad; j += kTopkThreads) {
-      uint32_t digit = 0xffffffffu;                       // sentinel: not a candidate
-      if (j < n_own) {
-        const uint32_t key = cached ? keys[j] : order_key(x[j0 + j]);
-        if ((key & hi_mask) == prefix) digit = (key >> shift) & digit_mask;
-      }
-      // one shared-memory atomic per distinct digit in the warp (scores of one head share
-      // their exponent, so in the first pass most lanes hit the same bin)
-      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sm.hist[digit], __popc(peers));
+    const int n_scan = listed ? (int)sm.n_cand : n_own;
+    for (int j = tid; j < n_scan; j += kTopkThreads) {
+      const uint32_t key = listed ? sm.cand[j] : (cached ? keys[j] : order_key(x[j0 + j]));
+      if ((key & hi_mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & digit_mask], 1u);
     }
     __syncthreads();
-    uint32_t* merged = leader_merged + pass * kBins;
-    for (int d = tid; d < kBins; d += kTopkThreads) {
+    // add the non-empty bins into every CTA's merged table; leave the local table clear
+    uint32_t local_bins[kBins / kTopkThreads];
+#pragma unroll
+    for (int e = 0; e < kBins / kTopkThreads; ++e) {
+      const int d = tid + e * kTopkThreads;
       const uint32_t c = sm.hist[d];
-      if (c) atomicAdd(merged + d, c);
+      local_bins[e] = c;
+      if (c) {
+        sm.hist[d] = 0u;
+#pragma unroll
+        for (int p = 0; p < kCluster; ++p) atomicAdd(peer_merged[p] + pass * kBins + d, c);
+      }
     }
     cluster.sync();
-    // every CTA scans the merged table from the top digit down; thread t owns digits
-    // 2047-2t and 2046-2t
+    // scan the merged table from the top digit down; thread t owns digits 2047-2t and 2046-2t
     const uint32_t remaining = sm.remaining;
     const int d_hi = kBins - 1 - 2 * tid;
-    const uint32_t v0 = merged[d_hi], v1 = merged[d_hi - 1];
+    const uint32_t v0 = sm.merged[pass][d_hi], v1 = sm.merged[pass][d_hi - 1];
     const uint32_t mine = v0 + v1;
     uint32_t incl = mine;
 #pragma unroll
@@ -117,17 +123,42 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
     }
     if (lane == 31) sm.warp_sum[warp] = incl;
     __syncthreads();
-    uint32_t before = 0u;
-    for (int w = 0; w < warp; ++w) before += sm.warp_sum[w];
-    incl += before;
+    if (warp == 0) {
+      const uint32_t ws = sm.warp_sum[lane];
+      uint32_t wi = ws;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += y;
+      }
+      sm.warp_sum[lane] = wi - ws;                         // exclusive prefix of the warp sums
+    }
+    __syncthreads();
+    incl += sm.warp_sum[warp];
     const uint32_t excl = incl - mine;
-    __syncthreads();                                       // prefix / remaining were read by everyone
     if (excl < remaining && incl >= remaining) {           // exactly one thread
       const bool first = excl + v0 >= remaining;
       sm.prefix = prefix | ((uint32_t)(first ? d_hi : d_hi - 1) << shift);
       sm.remaining = remaining - excl - (first ? 0u : v0);
     }
     __syncthreads();
+    if (pass == 0) {
+      // keep only this CTA's keys of the selected bin, if they fit the list (their number is
+      // this CTA's own count of that bin, which the owner of the bin still holds)
+      const uint32_t digit0 = sm.prefix >> 21;
+#pragma unroll
+      for (int e = 0; e < kBins / kTopkThreads; ++e)
+        if ((uint32_t)(tid + e * kTopkThreads) == digit0) sm.n_cand = local_bins[e] <= (uint32_t)kMaxCand ? 0u : 0xffffffffu;
+      __syncthreads();
+      listed = sm.n_cand == 0u;
+      if (listed) {
+        for (int j = tid; j < n_own; j += kTopkThreads) {
+          const uint32_t key = cached ? keys[j] : order_key(x[j0 + j]);
+          if ((key >> 21) == digit0) sm.cand[atomicAdd(&sm.n_cand, 1u)] = key;
+        }
+      }
+      __syncthreads();
+    }
   }
 
   const uint32_t thr = sm.prefix;          // key of the K-th largest score
@@ -151,14 +182,14 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
       g += __shfl_xor_sync(0xffffffffu, g, o);
       e += __shfl_xor_sync(0xffffffffu, e, o);
     }
-    if (lane == 0) { sm.cta_gt = g; sm.cta_eq = e; }
+    if (lane < kCluster) {                                 // lane p tells CTA p this CTA's totals
+      *cluster.map_shared_rank(&sm.peer_gt[rank], lane) = g;
+      *cluster.map_shared_rank(&sm.peer_eq[rank], lane) = e;
+    }
   }
-  cluster.sync();
+  cluster.sync();                    // the last remote access of the kernel is behind every CTA
   uint32_t gt_before = 0u, eq_before = 0u;
-  for (int r = 0; r < rank; ++r) {
-    gt_before += *cluster.map_shared_rank(&sm.cta_gt, r);
-    eq_before += *cluster.map_shared_rank(&sm.cta_eq, r);
-  }
+  for (int r = 0; r < rank; ++r) { gt_before += sm.peer_gt[r]; eq_before += sm.peer_eq[r]; }
   for (int w = 0; w < warp; ++w) { gt_before += sm.cnt_gt[w]; eq_before += sm.cnt_eq[w]; }
   uint32_t pos = gt_before + min(eq_before, n_ties);
   const uint32_t lt_mask = (1u << lane) - 1u;
@@ -173,7 +204,6 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
     pos += __popc(take_bal);
     eq_before += __popc(eq_bal);
   }
-  cluster.sync();                    // no CTA exits while another may still read its counts
 }
 
 }  // namespace
