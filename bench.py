@@ -42,7 +42,12 @@ FALLBACK_BF16_TFLOPS = 1590.0
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/ (bytes; None = not captured for that pair).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/evict_kernels_llama3_8b_32k.md (a 2-layer run of the same command; traffic per launch does not
+    # depend on the number of layers)
+    ("sweep1", "llama3_8b_32k"): 68345088 + 932608,
+    ("sweep2", "llama3_8b_32k"): 68804096 + 924160,
+}
 
 
 def load_peaks():
