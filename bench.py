@@ -198,6 +198,22 @@ def run_reference(args, w: gi.Workload):
     }))
 
 
+# ---------------------------------------------------------------------------- rank bookkeeping
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's device time (every rank runs its own replica of the workload)."""
+    if world == 1:
+        return float(ms)
+    import torch.distributed as dist
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(world: int, tokens: int, n_layers: int, ms_step: float) -> float:
+    """Tokens scored and evicted per second per layer over all ranks (weak scaling)."""
+    return world * tokens * n_layers / (ms_step * 1e-3)
+
+
 # ---------------------------------------------------------------------------------- GPU arm
 def run_ours(args, w: gi.Workload):
     import torch.distributed as dist
@@ -279,13 +295,10 @@ def run_ours(args, w: gi.Workload):
     dq.dapq_profile(ctx, False)
     clocks = sampler.stop() if sampler else None
 
-    if world > 1:
-        tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     tokens = w.total_prompt
-    value = world * tokens * n_layers / (ms_step * 1e-3)
+    value = whole_job_value(world, tokens, n_layers, ms_step)
 
     # ---- roofline of the dominant kernel
     kinds = {k: v for k, v in prof.items() if v[1] > 0}
@@ -338,14 +351,11 @@ def run_ours(args, w: gi.Workload):
         e1.record()
         barrier()
         ms_e2e = e0.elapsed_time(e1) / e2e_steps
-        if world > 1:
-            tt = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_e2e = float(tt.item())
+        ms_e2e = max_over_ranks(ms_e2e, world, dev)
         eb = 2 if w.dtype == "bf16" else 4
         h2d = n_layers * (2 * w.n_kv_heads * w.total_rows * w.head_dim * eb + w.batch * w.n_q_heads * w.n_pseudo * w.head_dim * eb)
         d2h = n_layers * (2 * w.n_kv_heads * KT * w.head_dim * eb + 4 * w.n_kv_heads * KT)
-        e2e = {"value": world * tokens * n_layers / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_value(world, tokens, n_layers, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps,
                "api": "dapq_evict_host (pinned host K/V/q in, compacted K/V + indices out, per layer)"}
 

@@ -42,7 +42,7 @@ struct TopkSmem {
   uint32_t warp_sum[kWarps];
   uint32_t cnt_gt[kWarps], cnt_eq[kWarps];
   uint32_t peer_gt[kCluster], peer_eq[kCluster];   // totals of every CTA of the cluster, pushed by their owners
-  uint32_t prefix, remaining, n_cand;
+  uint32_t prefix, remaining, n_cand, list_ok;
 };
 
 __global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kTopkThreads)
@@ -148,9 +148,9 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
       const uint32_t digit0 = sm.prefix >> 21;
 #pragma unroll
       for (int e = 0; e < kBins / kTopkThreads; ++e)
-        if ((uint32_t)(tid + e * kTopkThreads) == digit0) sm.n_cand = local_bins[e] <= (uint32_t)kMaxCand ? 0u : 0xffffffffu;
+        if ((uint32_t)(tid + e * kTopkThreads) == digit0) sm.list_ok = local_bins[e] <= (uint32_t)kMaxCand;
       __syncthreads();
-      listed = sm.n_cand == 0u;
+      listed = sm.list_ok != 0u;           // (a flag of its own: n_cand starts to move as soon as the first thread lists)
       if (listed) {
         for (int j = tid; j < n_own; j += kTopkThreads) {
           const uint32_t key = cached ? keys[j] : order_key(x[j0 + j]);

@@ -192,6 +192,11 @@ def test_topk_exact_with_ties(dq, lens, keep):
         for h in range(3):
             ref = orc.topk_select(s[h, w.cu_prompt[b]:w.cu_prompt[b + 1]].astype(np.float64), keep[b])
             np.testing.assert_array_equal(got[h, w.cu_keep[b]:w.cu_keep[b + 1]], ref, err_msg=f"b={b} h={h}")
+    # the select is integer work in a fixed order: every repeat gives the same indices
+    for _ in range(20):
+        again = torch.full_like(idx, -1)
+        dq.dapq_topk_select(ctx, torch.from_numpy(s).cuda(), w.cu_prompt, keep, again)
+        assert torch.equal(again, idx)
     dq.dapq_destroy(ctx)
 
 
@@ -293,3 +298,42 @@ def test_argument_errors_launch_nothing(dq):
         dq.dapq_topk_select(ctx, scores, [0, 100], [0], torch.empty(8, 10, dtype=torch.int32, device="cuda"))
     assert dq.dapq_launch_count(ctx) == n0
     dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------------ full-size configurations, sampled heads
+@pytest.mark.parametrize("name,heads", [("llama3_8b_32k", (0, 3, 7)), ("qwen25_7b_128k", (2,)),
+                                        ("batched_serving", (5,)), ("llama3_70b_128k", (6,))])
+def test_evict_full_size_sampled_heads(dq, name, heads):
+    """One layer of each benchmark configuration at its full size, through dapq_evict exactly as
+    bench.py launches it; the oracle checks the sampled KV heads (all sequences of the batch)."""
+    w = gi.workload(name)
+    data = gi.draw_layer(w, 0, "cuda")
+    ctx = _ctx(dq, w)
+    # structure is planted with the library's own rotation, as in the benchmark
+    q_rot = torch.empty_like(data["q_pre"])
+    dq.dapq_rope_pseudo_q(ctx, data["q_pre"], list(w.prompt_lens), q_rot)
+    torch.cuda.synchronize()
+    gi.plant_structure(w, data, q_rot)
+    got = _gpu_evict(dq, w, data, ctx)
+    dq.dapq_destroy(ctx)
+    G, N = w.group, w.n_pseudo
+    cu_p, cu_k, cu_r = w.cu_prompt, w.cu_keep, w.cu_rows
+    q64 = util.to_f64(data["q_pre"])
+    for h in heads:
+        k_h = data["k"][h].cpu()
+        v_h = data["v"][h].cpu()
+        k64 = util.to_f64(k_h)
+        for b in range(w.batch):
+            L, r0 = w.prompt_lens[b], int(cu_r[b])
+            qr = orc.rope_pseudo_q(q64[b, h * G:(h + 1) * G], L, w.rope_base)
+            ref = orc.score_sequence(qr, k64[None, r0:r0 + L + N], L, G)["scores"][0]
+            ref_idx = orc.topk_select(ref, w.keep[b])
+            tag = f"{name} b={b} kvh={h}"
+            util.assert_scores_close(got["scores"][h, cu_p[b]:cu_p[b + 1]], ref, tag)
+            gidx = got["idx"][h, cu_k[b]:cu_k[b + 1]]
+            util.assert_index_sets_match(gidx, ref, ref_idx, L, tag)
+            rows = torch.as_tensor(gidx.astype(np.int64) + r0)
+            assert torch.equal(got["k_out"][h, cu_k[b]:cu_k[b + 1]], k_h[rows]), tag
+            assert torch.equal(got["v_out"][h, cu_k[b]:cu_k[b + 1]], v_h[rows]), tag
+            for p in (data["needle_pos"][b, h] if w.n_needles else []):
+                assert int(p) in set(gidx.tolist()), f"{tag}: planted needle {p} evicted"
