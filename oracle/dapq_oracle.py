@@ -125,6 +125,28 @@ def score_sequence(q_rot: np.ndarray, k_seq: np.ndarray, prompt_len: int, group:
 
 
 # --------------------------------------------------------------------------------------
+# Optional pooling of the accumulated scores before selection.  The paper specifies none
+# for DapQ; it describes the SnapKV / PyramidKV baselines as selecting on pooled accumulated
+# attention scores (Sections 2 and 5.1), which this option reproduces.
+# --------------------------------------------------------------------------------------
+def pool_scores(scores: np.ndarray, kernel: int, mode: str) -> np.ndarray:
+    """1-D pooling along one sequence's prompt positions: window of odd width `kernel`
+    centred on each position, stride 1, clipped at the ends of the sequence.
+    mode "max": largest score in the window; "avg": mean of the scores in the window
+    (of the positions that exist, so the ends average fewer values); "none": unchanged."""
+    s = np.asarray(scores, dtype=np.float64)
+    if mode == "none" or kernel <= 1:
+        return s.copy()
+    assert kernel % 2 == 1 and mode in ("max", "avg")
+    L, r = s.shape[-1], kernel // 2
+    out = np.empty_like(s)
+    for j in range(L):
+        win = s[..., max(0, j - r):min(L, j + r + 1)]
+        out[..., j] = win.max(axis=-1) if mode == "max" else win.mean(axis=-1)
+    return out
+
+
+# --------------------------------------------------------------------------------------
 # Section 4.2, Eq. 5: M_retain = TopK_j S(j)
 # --------------------------------------------------------------------------------------
 def topk_select(scores: np.ndarray, k_keep: int) -> np.ndarray:
@@ -152,12 +174,15 @@ def compact_kv(k_seq_head: np.ndarray, v_seq_head: np.ndarray,
 def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int],
           prompt_len: Sequence[int], k_keep: Sequence[int], rope_base: float,
           scale: Optional[float] = None,
-          pos_start: Optional[Sequence[int]] = None) -> Dict[str, object]:
+          pos_start: Optional[Sequence[int]] = None, pool_mode: str = "none",
+          pool_kernel: int = 1) -> Dict[str, object]:
     """The whole path for one layer (Figure 1): rotate, score, select, compact.
 
     q_pre [B, H_q, N, d] pre-RoPE pseudo queries (any float dtype; converted exactly
     to float64); k, v [H_kv, R, d] packed cache whose sequence b owns rows
     cu_rows[b] .. cu_rows[b+1] (L_b prompt rows, then N synthetic rows).
+    With pool_mode "max" / "avg" the selection runs on the pooled scores (returned as
+    "pooled"); "scores" are always the unpooled Eq. 4 sums.
     Returns per-sequence lists: scores [H_kv, L_b], idx [H_kv, K_b] (sequence-local),
     k_out / v_out [H_kv, K_b, d] in the dtype of k / v, plus lse and the two masses.
     """
@@ -165,7 +190,7 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
     Hkv = k.shape[0]
     G = Hq // Hkv
     out: Dict[str, List] = {key: [] for key in
-                            ("q_rot", "scores", "lse", "prompt_mass", "syn_mass",
+                            ("q_rot", "scores", "pooled", "lse", "prompt_mass", "syn_mass",
                              "idx", "k_out", "v_out")}
     for b in range(B):
         L = int(prompt_len[b])
@@ -177,13 +202,15 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
         v_seq = v[:, r0:r0 + L + n]
         res = score_sequence(q_rot, k_seq, L, G, scale)
         kk = min(int(k_keep[b]), L)
-        idx = np.stack([topk_select(res["scores"][h], kk) for h in range(Hkv)])
+        pooled = pool_scores(res["scores"], pool_kernel, pool_mode)
+        idx = np.stack([topk_select(pooled[h], kk) for h in range(Hkv)])
         kept = [compact_kv(k_seq[h], v_seq[h], idx[h]) for h in range(Hkv)]
         ko = np.stack([kv[0] for kv in kept])
         vo = np.stack([kv[1] for kv in kept])
         out["q_rot"].append(q_rot)
         for key in ("scores", "lse", "prompt_mass", "syn_mass"):
             out[key].append(res[key])
+        out["pooled"].append(pooled)
         out["idx"].append(idx)
         out["k_out"].append(ko)
         out["v_out"].append(vo)

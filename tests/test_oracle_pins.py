@@ -305,3 +305,39 @@ def test_planted_needles_are_retained():
         for p in data["needle_pos"][0, h]:
             assert int(p) in idx
             assert sc[p] >= 10 * kth
+
+
+# ------------------------------------------------------------------ optional pooling
+@pytest.mark.parametrize("L,kernel", [(1, 3), (2, 5), (7, 7), (50, 5), (33, 13)])
+def test_pooling_matches_library_pooling(L, kernel):
+    s = np.abs(_rand((3, L), 30)) + 0.1
+    t = torch.from_numpy(s)[None]
+    r = kernel // 2
+    # max: the library pads with -inf, which is clipping the window
+    lib_max = torch.nn.functional.max_pool1d(t, kernel, stride=1, padding=r)[0].numpy()
+    np.testing.assert_array_equal(orc.pool_scores(s, kernel, "max"), lib_max)
+    # avg over the positions that exist = the library's count_include_pad=False
+    lib_avg = torch.nn.functional.avg_pool1d(t, kernel, stride=1, padding=r, count_include_pad=False)[0].numpy()
+    np.testing.assert_allclose(orc.pool_scores(s, kernel, "avg"), lib_avg, rtol=1e-13)
+
+
+def test_pooling_hand_case_and_identity():
+    s = np.array([1.0, 5.0, 2.0, 0.0, 3.0])
+    np.testing.assert_array_equal(orc.pool_scores(s, 3, "max"), [5, 5, 5, 3, 3])
+    np.testing.assert_allclose(orc.pool_scores(s, 3, "avg"), [3.0, 8 / 3, 7 / 3, 5 / 3, 1.5])
+    np.testing.assert_array_equal(orc.pool_scores(s, 1, "max"), s)
+    np.testing.assert_array_equal(orc.pool_scores(s, 7, "none"), s)
+
+
+def test_evict_selects_on_pooled_scores():
+    rng = np.random.default_rng(31)
+    q = rng.standard_normal((1, 2, 4, 16))
+    k = rng.standard_normal((1, 40 + 4, 16))
+    plain = orc.evict(q, k, k, [0, 44], [40], [6], 1.0e4)
+    pooled = orc.evict(q, k, k, [0, 44], [40], [6], 1.0e4, pool_mode="max", pool_kernel=5)
+    np.testing.assert_array_equal(pooled["scores"][0], plain["scores"][0])      # Eq. 4 sums are untouched
+    np.testing.assert_array_equal(pooled["pooled"][0], orc.pool_scores(plain["scores"][0], 5, "max"))
+    np.testing.assert_array_equal(pooled["idx"][0][0], orc.topk_select(pooled["pooled"][0][0], 6))
+    # max pooling spreads the top score over its window: its neighbours are kept (ties -> lower index)
+    top = int(np.argmax(plain["scores"][0][0]))
+    assert {max(0, top - 2), top}.issubset(set(pooled["idx"][0][0].tolist()))
