@@ -66,12 +66,14 @@ typedef enum {
 
 typedef enum { DAPQ_BF16 = 0, DAPQ_F32 = 1 } dapq_dtype;
 
-enum { DAPQ_MAX_BATCH = 128, DAPQ_MAX_PSEUDO = 128, DAPQ_HEAD_DIM = 128 };
+enum { DAPQ_MAX_BATCH = 128, DAPQ_MAX_PSEUDO = 128, DAPQ_HEAD_DIM = 128, DAPQ_MAX_POOL_KERNEL = 127 };
 
 /* Pooling of the accumulated scores before selection.  The paper specifies none for
  * DapQ (it mentions pooling only for the SnapKV / PyramidKV baselines), so NONE is the
- * default; MAX / AVG apply a 1-D window of odd width pool_kernel, stride 1, clipped at
- * the ends of each sequence. */
+ * default; MAX / AVG apply a 1-D window of odd width pool_kernel (3 .. DAPQ_MAX_POOL_KERNEL),
+ * stride 1, clipped at the ends of each sequence (AVG is the mean of the positions that
+ * exist).  With pooling on, dapq_topk_select and dapq_evict select on the pooled scores;
+ * the scores that dapq_score and dapq_evict hand out are always the unpooled Eq. 4 sums. */
 typedef enum { DAPQ_POOL_NONE = 0, DAPQ_POOL_MAX = 1, DAPQ_POOL_AVG = 2 } dapq_pool_mode;
 
 /* dapq_shape.flags.  DAPQ_FLAG_CUDA_CORE_SCORER keeps the scorer on the CUDA-core kernels
@@ -133,7 +135,7 @@ DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
  * enabled.  ms_out / count_out: host [DAPQ_PROF_KINDS], in the order of dapq_prof_kind. */
 typedef enum {
   DAPQ_PROF_ROPE = 0, DAPQ_PROF_SWEEP1 = 1, DAPQ_PROF_LSE_MERGE = 2, DAPQ_PROF_SWEEP2 = 3,
-  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_KINDS = 6
+  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_POOL = 6, DAPQ_PROF_KINDS = 7
 } dapq_prof_kind;
 DAPQ_API dapq_status dapq_profile(dapq_ctx* ctx, int32_t enable);
 DAPQ_API dapq_status dapq_profile_read(dapq_ctx* ctx, void* stream, double* ms_out, int64_t* count_out);
@@ -160,7 +162,8 @@ DAPQ_API dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cac
 /* Section 4.2, Eq. 5: for every (b, kvh) the min(K_b, L_b) positions with the largest
  * score; equal scores at the threshold go to the lower position; positions are written
  * in ascending order.  scores: device [H_kv, T] (finite, >= 0); cu_prompt_host: host
- * [B+1]; k_keep_host: host [B], K_b >= 1; idx_out: device [H_kv, KT]. */
+ * [B+1]; k_keep_host: host [B], K_b >= 1; idx_out: device [H_kv, KT].  If the context was
+ * created with a pooling mode, the scores are pooled first (into the workspace). */
 DAPQ_API dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* cu_prompt_host,
                              const int32_t* k_keep_host, int32_t batch, int32_t* idx_out,
                              void* stream);

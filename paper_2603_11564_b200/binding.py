@@ -170,7 +170,7 @@ def dapq_launch_count(ctx) -> int:
     return int(load_library().dapq_launch_count(ctx))
 
 
-PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact")
+PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact", "pool")
 
 
 def dapq_profile(ctx, enable: bool) -> None:

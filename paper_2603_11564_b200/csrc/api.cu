@@ -213,6 +213,21 @@ dapq_status run_score(dapq_ctx* ctx, int q_dtype, const void* q_rot, const Cache
   return DAPQ_OK;
 }
 
+// Eq. 5 on the scores, or on their pooled image if the context asks for pooling.
+dapq_status run_select(dapq_ctx* ctx, const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
+                       const SeqTable& t, cudaStream_t s) {
+  cudaError_t e;
+  if (ctx->shape.pool_mode != DAPQ_POOL_NONE) {
+    e = launch_pool(scores, ctx->pooled, score_stride, t, ctx->dims.n_kv_heads, ctx->shape.pool_kernel,
+                    ctx->shape.pool_mode, s, &ctx->log);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "pooling kernel");
+    scores = ctx->pooled;
+  }
+  e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &ctx->log);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
+  return DAPQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -238,7 +253,10 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
     return bail(DAPQ_ERR_UNSUPPORTED, "max_batch > 128 or max_total_rows >= 2^31");
   if (sh->dtype != DAPQ_BF16 && sh->dtype != DAPQ_F32) return bail(DAPQ_ERR_INVALID_ARG, "unknown dtype");
   if (sh->flags & ~DAPQ_FLAG_CUDA_CORE_SCORER) return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
-  if (sh->pool_mode != DAPQ_POOL_NONE) return bail(DAPQ_ERR_UNSUPPORTED, "pooling is not available");
+  if (sh->pool_mode != DAPQ_POOL_NONE && sh->pool_mode != DAPQ_POOL_MAX && sh->pool_mode != DAPQ_POOL_AVG)
+    return bail(DAPQ_ERR_INVALID_ARG, "unknown pool_mode");
+  if (sh->pool_mode != DAPQ_POOL_NONE && (sh->pool_kernel < 3 || sh->pool_kernel > DAPQ_MAX_POOL_KERNEL || sh->pool_kernel % 2 == 0))
+    return bail(DAPQ_ERR_UNSUPPORTED, "pool_kernel must be odd, 3 .. 127");
   if (!sh->inv_freq_host && !(sh->rope_base > 0.0)) return bail(DAPQ_ERR_INVALID_ARG, "rope_base must be > 0");
   if (!(sh->softmax_scale >= 0.f)) return bail(DAPQ_ERR_INVALID_ARG, "softmax_scale must be >= 0");
 
@@ -275,6 +293,8 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   ok = ok && cudaMalloc(&ctx->lse2, ((size_t)sh->max_batch * hq_n + 32) * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->scores, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->idx, (size_t)sh->n_kv_heads * rows * sizeof(int32_t)) == cudaSuccess;
+  if (sh->pool_mode != DAPQ_POOL_NONE)
+    ok = ok && cudaMalloc(&ctx->pooled, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMemcpy(ctx->inv_freq, freq, sizeof(freq), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemset(ctx->status, 0, sizeof(int)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); return bail(DAPQ_ERR_CUDA, "workspace allocation failed"); }
@@ -386,10 +406,7 @@ dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const int32_t* 
   dapq_status st = build_table(ctx, batch, nullptr, nullptr, cu_prompt_host, k_keep_host, nullptr, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  cudaError_t e = launch_topk(scores, t.cu_prompt[batch], idx_out, t.cu_keep[batch], t, ctx->dims.n_kv_heads,
-                              (cudaStream_t)stream, &ctx->log);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
-  return DAPQ_OK;
+  return run_select(ctx, scores, t.cu_prompt[batch], idx_out, t.cu_keep[batch], t, (cudaStream_t)stream);
 }
 
 dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const int32_t* idx,
@@ -443,8 +460,8 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
     st = run_score(ctx, DAPQ_F32, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
   }
   if (st != DAPQ_OK) return st;
-  e = launch_topk(scores, score_stride, idx, idx_stride, t, ctx->dims.n_kv_heads, s, &ctx->log);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "top-k kernel");
+  st = run_select(ctx, scores, score_stride, idx, idx_stride, t, s);
+  if (st != DAPQ_OK) return st;
   e = launch_compact(ctx->shape.dtype, cd, idx, idx_stride, k_out, v_out, t, ctx->dims.n_kv_heads, ctx->status, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "compaction kernel");
   return DAPQ_OK;

@@ -63,7 +63,7 @@ __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
 }
 
 // Kernel kinds, for launch accounting and the optional per-kernel event timing.
-enum KernelKind : int { kKindRope = 0, kKindSweep1, kKindLseMerge, kKindSweep2, kKindTopk, kKindCompact,
+enum KernelKind : int { kKindRope = 0, kKindSweep1, kKindLseMerge, kKindSweep2, kKindTopk, kKindCompact, kKindPool,
                         kKindCount };
 
 // Counts launches and, while profiling is on, brackets every launch with CUDA events on
@@ -110,6 +110,10 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log);
+
+// pooled[kvh, j] = max / mean of scores[kvh, j - kernel/2 .. j + kernel/2] within each sequence.
+cudaError_t launch_pool(const float* scores, float* pooled, int64_t stride, const SeqTable& t, int n_kv_heads,
+                        int kernel, int mode, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, int64_t idx_stride,
                            void* k_out, void* v_out, const SeqTable& t, int n_kv_heads, int* status,

@@ -337,3 +337,37 @@ def test_evict_full_size_sampled_heads(dq, name, heads):
             assert torch.equal(got["v_out"][h, cu_k[b]:cu_k[b + 1]], v_h[rows]), tag
             for p in (data["needle_pos"][b, h] if w.n_needles else []):
                 assert int(p) in set(gidx.tolist()), f"{tag}: planted needle {p} evicted"
+
+
+# ------------------------------------------------------------------ optional pooling
+@pytest.mark.parametrize("mode,kernel", [("max", 7), ("avg", 5), ("max", 127), ("avg", 3)])
+def test_pooled_selection_matches_oracle(dq, mode, kernel):
+    code = dq.DAPQ_POOL_MAX if mode == "max" else dq.DAPQ_POOL_AVG
+    w = gi.scaled_down("batched_serving", 16, n_layers=1)
+    data = util.make_case(w)
+    ref = orc.evict(util.to_f64(data["q_pre"]), util.to_f64(data["k"]), util.to_f64(data["v"]), w.cu_rows,
+                    w.prompt_lens, w.keep, w.rope_base, pool_mode=mode, pool_kernel=kernel)
+    ctx = _ctx(dq, w, pool_mode=code, pool_kernel=kernel)
+    got = _gpu_evict(dq, w, data, ctx)
+    cu_p, cu_k, cu_r = w.cu_prompt, w.cu_keep, w.cu_rows
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            tag = f"pool {mode}{kernel} b={b} kvh={h}"
+            # the scores handed out stay the unpooled Eq. 4 sums
+            util.assert_scores_close(got["scores"][h, cu_p[b]:cu_p[b + 1]], ref["scores"][b][h], tag)
+            gidx = got["idx"][h, cu_k[b]:cu_k[b + 1]]
+            util.assert_index_sets_match(gidx, ref["pooled"][b][h], ref["idx"][b][h], w.prompt_lens[b], tag)
+            rows = torch.as_tensor(gidx.astype(np.int64) + int(cu_r[b]))
+            assert torch.equal(got["k_out"][h, cu_k[b]:cu_k[b + 1]], data["k"][h].cpu()[rows]), tag
+    # dapq_topk_select alone pools too: max pooling of fp32 scores is exact, so the sets are equal
+    if mode == "max":
+        rng = np.random.default_rng(9)
+        s = rng.random((w.n_kv_heads, w.total_prompt)).astype(np.float32)
+        idx = torch.empty((w.n_kv_heads, int(cu_k[-1])), dtype=torch.int32, device="cuda")
+        dq.dapq_topk_select(ctx, torch.from_numpy(s).cuda(), cu_p, w.keep, idx)
+        torch.cuda.synchronize()
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                pooled = orc.pool_scores(s[h, cu_p[b]:cu_p[b + 1]].astype(np.float64), kernel, "max")
+                np.testing.assert_array_equal(idx[h, cu_k[b]:cu_k[b + 1]].cpu().numpy(), orc.topk_select(pooled, w.keep[b]))
+    dq.dapq_destroy(ctx)
