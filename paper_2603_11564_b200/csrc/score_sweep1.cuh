@@ -37,8 +37,8 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-      s0 += ex2(fmaf(x[e], c, neg));
-      s1 += ex2(fmaf(x[e + 1], c, neg));
+      s0 += ex2_sel(fmaf(x[e], c, neg), e);
+      s1 += ex2_sel(fmaf(x[e + 1], c, neg), e + 1);
     }
     z += s0 + s1;
   }

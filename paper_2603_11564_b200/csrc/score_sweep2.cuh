@@ -97,16 +97,25 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * 2 * rows_pad + grow;
             const int64_t step = (int64_t)a.n_kv_heads * 2 * rows_pad;
             const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
-            float mx = -CUDART_INF_F;
-            for (int cc = 0; cc < nc; ++cc) {
-              mx = fmaxf(mx, p[cc * step].x);
-              mx = fmaxf(mx, p[cc * step + rows_pad].x);
-            }
-            float z = 0.f;
-            for (int cc = 0; cc < nc; ++cc) {
-              const float2 p0 = p[cc * step], p1 = p[cc * step + rows_pad];
-              z += p0.y * exp2f(p0.x - mx);
-              z += p1.y * exp2f(p1.x - mx);
+            // one pass, eight independent loads in flight; (max, sum) merged in chunk order
+            float mx = -CUDART_INF_F, z = 0.f;
+            for (int c0 = 0; c0 < nc; c0 += 4) {
+              float2 q[8];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const bool in = c0 + u < nc;
+                q[2 * u] = in ? __ldg(p + (c0 + u) * step) : make_float2(-CUDART_INF_F, 0.f);
+                q[2 * u + 1] = in ? __ldg(p + (c0 + u) * step + rows_pad) : make_float2(-CUDART_INF_F, 0.f);
+              }
+              float m8 = q[0].x;
+#pragma unroll
+              for (int u = 1; u < 8; ++u) m8 = fmaxf(m8, q[u].x);
+              if (m8 > mx) {
+                z *= exp2f(mx - m8);                        // exp2f(-inf) = 0 on the first chunk
+                mx = m8;
+              }
+#pragma unroll
+              for (int u = 0; u < 8; ++u) z += q[u].y * exp2f(q[u].x - mx);
             }
             l2 = mx + log2f(z);
           }
@@ -138,10 +147,10 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
               for (int e = 0; e < 32; e += 4) {
                 const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
-                sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, -l4.x));
-                sum1 += ex2(fmaf(__uint_as_float(v[k & 1][e + 1]), c, -l4.y));
-                sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e + 2]), c, -l4.z));
-                sum1 += ex2(fmaf(__uint_as_float(v[k & 1][e + 3]), c, -l4.w));
+                sum0 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e]), c, -l4.x), e);
+                sum1 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 1]), c, -l4.y), e + 1);
+                sum0 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 2]), c, -l4.z), e + 2);
+                sum1 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 3]), c, -l4.w), e + 3);
               }
             } else {
 #pragma unroll

@@ -125,6 +125,31 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x on the FMA / ALU pipes instead of the MUFU: round-to-nearest split x = n + f with the
+// 1.5 * 2^23 trick, a degree-3 minimax polynomial for 2^f on [-0.5, 0.5] (relative error below
+// 7.5e-5), and n added into the exponent field.  Inputs below -125 give 2^-125.  The scorer's
+// epilogues owe one exponential per (query, key) pair and the MUFU pipe delivers only 16 per
+// clock and SM, so every kPolyEvery-th element of a piece takes this path.
+#ifndef DAPQ_POLY_EVERY
+#define DAPQ_POLY_EVERY 4
+#endif
+constexpr int kPolyEvery = DAPQ_POLY_EVERY;
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -125.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.0551716648f, f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+// The e-th element of a 32-column piece (e is a constant after unrolling): polynomial for
+// every kPolyEvery-th one, MUFU otherwise; kPolyEvery = 0 keeps everything on the MUFU.
+__device__ __forceinline__ float ex2_sel(float x, int e) {
+  if (kPolyEvery > 0 && (e % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery > 0 ? kPolyEvery : 1) - 1) return ex2_poly(x);
+  return ex2(x);
+}
+
 // Three-input maximum (one instruction on sm_100).
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
