@@ -1,6 +1,7 @@
 // Per-head selection of the retained tokens (Section 4.2, Eq. 5: M_retain = TopK_j S(j)).
 //
-// One thread-block cluster of 8 CTAs per (sequence, KV head).  Each CTA owns a contiguous
+// One thread-block cluster of 1, 2, 4 or 8 CTAs (by the longest sequence: 4k to 16k keys per
+// CTA, fewer CTAs when the grid would not fit one wave) per (sequence, KV head).  Each CTA owns a contiguous
 // slice of the head's scores and keeps their order-preserving integer images in shared
 // memory, so the scores are read from global memory once.  A 3-pass radix select (11 + 11 +
 // 10 bits, most significant first) finds the exact bit pattern of the K-th largest score and
@@ -24,7 +25,9 @@ namespace {
 
 constexpr int kTopkThreads = 1024;
 constexpr int kWarps = kTopkThreads / 32;
-constexpr int kCluster = 8;                   // CTAs per (sequence, head); portable cluster size
+constexpr int kCluster = 8;                   // most CTAs per (sequence, head); portable cluster size
+constexpr int kKeysPerCta = 4096;             // a CTA owns about this many keys, twice or four times as many
+constexpr int kWaveCtas = 296;                // when the grid would otherwise exceed one wave (2 CTAs per SM)
 constexpr int kBins = 2048;                   // 11-bit digits (the last pass uses 1024 of them)
 constexpr int kMaxSliceSmem = 36864;          // keys a CTA can cache (144 KB); longer slices re-read global
 constexpr int kMaxCand = 4096;                // candidate keys a CTA lists after the first pass
@@ -45,7 +48,7 @@ struct TopkSmem {
   uint32_t prefix, remaining, n_cand, list_ok;
 };
 
-__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kTopkThreads)
+__global__ void __launch_bounds__(kTopkThreads)
 topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32_t* __restrict__ idx,
                    int64_t idx_stride, const __grid_constant__ SeqTable t, int cache_keys) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -54,7 +57,8 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
 
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
-  const int b = blockIdx.x / kCluster, kvh = blockIdx.y;
+  const int n_cta = (int)cluster.num_blocks();               // CTAs of this cluster (1, 2, 4 or 8)
+  const int b = blockIdx.x / n_cta, kvh = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int L = t.prompt_len[b];
   const int K = t.cu_keep[b + 1] - t.cu_keep[b];
@@ -62,7 +66,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
   int32_t* out = idx + (int64_t)kvh * idx_stride + t.cu_keep[b];
 
   // slice of this CTA: [j0, j1), a multiple of 32 keys long so that warps stay converged
-  const int slice = (((L + kCluster - 1) / kCluster) + 31) & ~31;
+  const int slice = (((L + n_cta - 1) / n_cta) + 31) & ~31;
   const int j0 = min(L, rank * slice), j1 = min(L, j0 + slice);
   const int n_own = j1 - j0;
 
@@ -82,7 +86,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
 
   uint32_t* peer_merged[kCluster];
 #pragma unroll
-  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&sm.merged[0][0], p);
+  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&sm.merged[0][0], p < n_cta ? p : 0);
   bool listed = false;               // the later passes read the candidate list instead of the slice
 
   for (int pass = 0; pass < 3; ++pass) {
@@ -106,7 +110,8 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
       if (c) {
         sm.hist[d] = 0u;
 #pragma unroll
-        for (int p = 0; p < kCluster; ++p) atomicAdd(peer_merged[p] + pass * kBins + d, c);
+        for (int p = 0; p < kCluster; ++p)
+          if (p < n_cta) atomicAdd(peer_merged[p] + pass * kBins + d, c);
       }
     }
     cluster.sync();
@@ -182,7 +187,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
       g += __shfl_xor_sync(0xffffffffu, g, o);
       e += __shfl_xor_sync(0xffffffffu, e, o);
     }
-    if (lane < kCluster) {                                 // lane p tells CTA p this CTA's totals
+    if (lane < n_cta) {                                    // lane p tells CTA p this CTA's totals
       *cluster.map_shared_rank(&sm.peer_gt[rank], lane) = g;
       *cluster.map_shared_rank(&sm.peer_eq[rank], lane) = e;
     }
@@ -212,17 +217,31 @@ cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log) {
   int max_len = 1;
   for (int b = 0; b < t.batch; ++b) max_len = t.prompt_len[b] > max_len ? t.prompt_len[b] : max_len;
-  const int slice = (((max_len + kCluster - 1) / kCluster) + 31) & ~31;
+  int n_cta = 1;
+  while (n_cta < kCluster && (int64_t)n_cta * kKeysPerCta < max_len) n_cta *= 2;
+  while (n_cta > 1 && t.batch * n_kv_heads * n_cta > kWaveCtas && (int64_t)(n_cta / 2) * 4 * kKeysPerCta >= max_len) n_cta /= 2;
+  const int slice = (((max_len + n_cta - 1) / n_cta) + 31) & ~31;
   const int cache_keys = slice <= kMaxSliceSmem ? slice : 0;          // 0: every pass re-reads global memory
   const size_t smem = sizeof(TopkSmem) + (size_t)cache_keys * sizeof(uint32_t);
   cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)(sizeof(TopkSmem) + (size_t)kMaxSliceSmem * sizeof(uint32_t)));
   if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(t.batch * n_cta, n_kv_heads);
+  cfg.blockDim = dim3(kTopkThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_cta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   log->begin(kKindTopk, s);
-  topk_select_kernel<<<dim3(t.batch * kCluster, n_kv_heads), kTopkThreads, smem, s>>>(scores, score_stride, idx,
-                                                                                      idx_stride, t, cache_keys);
+  e = cudaLaunchKernelEx(&cfg, topk_select_kernel, scores, score_stride, idx, idx_stride, t, cache_keys);
   log->end(s);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace dapq
