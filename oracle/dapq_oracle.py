@@ -171,6 +171,16 @@ def compact_kv(k_seq_head: np.ndarray, v_seq_head: np.ndarray,
     return k_seq_head[idx].copy(), v_seq_head[idx].copy()
 
 
+# --------------------------------------------------------------------------------------
+# Section 3.3, Eq. 1-3: recall of a predicted retained set against a gold one
+# --------------------------------------------------------------------------------------
+def recall(idx_gold: np.ndarray, idx_pred: np.ndarray) -> float:
+    """|M_gold ∩ M_pred| / |M_gold| for two index sets of one head (Eq. 3)."""
+    gold = set(int(x) for x in np.asarray(idx_gold).ravel())
+    pred = set(int(x) for x in np.asarray(idx_pred).ravel())
+    return len(gold & pred) / len(gold)
+
+
 def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int],
           prompt_len: Sequence[int], k_keep: Sequence[int], rope_base: float,
           scale: Optional[float] = None,

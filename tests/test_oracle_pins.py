@@ -341,3 +341,29 @@ def test_evict_selects_on_pooled_scores():
     # max pooling spreads the top score over its window: its neighbours are kept (ties -> lower index)
     top = int(np.argmax(plain["scores"][0][0]))
     assert {max(0, top - 2), top}.issubset(set(pooled["idx"][0][0].tolist()))
+
+
+# ------------------------------------------------------------------ recall (Section 3.3)
+def test_recall_hand_cases_and_library_agreement():
+    assert orc.recall([1, 2, 3, 4], [1, 2, 3, 4]) == 1.0
+    assert orc.recall([1, 2, 3, 4], [5, 6, 7, 8]) == 0.0
+    assert orc.recall([0, 2, 4, 6], [1, 2, 3, 4]) == 0.5            # {2, 4} of four gold tokens
+    rng = np.random.default_rng(40)
+    for _ in range(5):
+        a = np.sort(rng.choice(500, 60, replace=False))
+        b = np.sort(rng.choice(500, 60, replace=False))
+        assert orc.recall(a, b) == pytest.approx(np.intersect1d(a, b).size / 60)
+
+
+def test_recall_of_a_smaller_window_against_a_larger_one():
+    # Eq. 1-3 on one cache: gold = top-K under all 16 queries, pred = top-K under the last 4;
+    # identical windows give 1, and the value is a fraction with denominator K
+    rng = np.random.default_rng(41)
+    q = rng.standard_normal((1, 1, 16, 16))
+    k = rng.standard_normal((1, 60 + 16, 16))
+    gold = orc.evict(q, k, k, [0, 76], [60], [10], 1.0e4)["idx"][0][0]
+    assert orc.recall(gold, gold) == 1.0
+    k4 = np.concatenate([k[:, :60], k[:, 72:]], axis=1)
+    pred = orc.evict(q[:, :, 12:], k4, k4, [0, 64], [60], [10], 1.0e4, pos_start=[72])["idx"][0][0]
+    r = orc.recall(gold, pred)
+    assert 0.0 <= r <= 1.0 and abs(r * 10 - round(r * 10)) < 1e-12
