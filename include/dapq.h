@@ -135,7 +135,7 @@ DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
  * enabled.  ms_out / count_out: host [DAPQ_PROF_KINDS], in the order of dapq_prof_kind. */
 typedef enum {
   DAPQ_PROF_ROPE = 0, DAPQ_PROF_SWEEP1 = 1, DAPQ_PROF_LSE_MERGE = 2, DAPQ_PROF_SWEEP2 = 3,
-  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_POOL = 6, DAPQ_PROF_KINDS = 7
+  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_POOL = 6, DAPQ_PROF_RECALL = 7, DAPQ_PROF_KINDS = 8
 } dapq_prof_kind;
 DAPQ_API dapq_status dapq_profile(dapq_ctx* ctx, int32_t enable);
 DAPQ_API dapq_status dapq_profile_read(dapq_ctx* ctx, void* stream, double* ms_out, int64_t* count_out);
@@ -174,6 +174,14 @@ DAPQ_API dapq_status dapq_topk_select(dapq_ctx* ctx, const float* scores, const 
  * skipped and flagged through dapq_poll_status as DAPQ_ERR_INVALID_ARG). */
 DAPQ_API dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const int32_t* idx,
                             const int32_t* k_keep_host, void* k_out, void* v_out, void* stream);
+
+/* Section 3.3, Eq. 1-3: Recall_W = |M_gold ∩ M_pred| / |M_gold| per (sequence, KV head), for two
+ * retained sets chosen with the same budgets on the same cache (e.g. a small observation window
+ * against a large one).  idx_gold, idx_pred: device [H_kv, KT] as written by dapq_topk_select
+ * (ascending within a sequence); recall_out: device [B, H_kv] fp32. */
+DAPQ_API dapq_status dapq_recall(dapq_ctx* ctx, const int32_t* idx_gold, const int32_t* idx_pred,
+                        const int32_t* prompt_len_host, const int32_t* k_keep_host, int32_t batch,
+                        float* recall_out, void* stream);
 
 /* Figure 1, the whole eviction step for one layer: rotate to positions L_b + i, score,
  * select, compact.  idx_out, scores_out may be NULL (kept in the workspace). */

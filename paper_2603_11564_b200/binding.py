@@ -27,7 +27,7 @@ _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORT
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
            "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
-           "dapq_compact_kv", "dapq_evict", "dapq_evict_host", "dapq_score_static")
+           "dapq_compact_kv", "dapq_evict", "dapq_evict_host", "dapq_score_static", "dapq_recall")
 
 
 class DapqError(RuntimeError):
@@ -90,6 +90,8 @@ def load_library() -> C.CDLL:
     lib.dapq_evict.restype = C.c_int
     lib.dapq_evict_host.argtypes = [vp, vp, C.POINTER(dapq_cache_view), i32p, vp, vp, vp, vp]
     lib.dapq_evict_host.restype = C.c_int
+    lib.dapq_recall.argtypes = [vp, vp, vp, i32p, i32p, C.c_int32, f32p, vp]
+    lib.dapq_recall.restype = C.c_int
     lib.dapq_score_static.argtypes = [C.POINTER(dapq_shape), C.c_int, vp, C.POINTER(dapq_cache_view), f32p, vp,
                                       C.c_char_p, C.c_size_t]
     lib.dapq_score_static.restype = C.c_int
@@ -170,7 +172,7 @@ def dapq_launch_count(ctx) -> int:
     return int(load_library().dapq_launch_count(ctx))
 
 
-PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact", "pool")
+PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact", "pool", "recall")
 
 
 def dapq_profile(ctx, enable: bool) -> None:
@@ -214,6 +216,14 @@ def dapq_compact_kv(ctx, k: torch.Tensor, v: torch.Tensor, cu_rows, prompt_len, 
     kk, kk_p = _i32(k_keep)
     _check(ctx, load_library().dapq_compact_kv(ctx, C.byref(view), idx.data_ptr(), kk_p, k_out.data_ptr(),
                                                v_out.data_ptr(), _stream(stream)))
+
+
+def dapq_recall(ctx, idx_gold: torch.Tensor, idx_pred: torch.Tensor, prompt_len, k_keep, recall_out: torch.Tensor,
+                stream=None) -> None:
+    pl, pl_p = _i32(prompt_len)
+    kk, kk_p = _i32(k_keep)
+    _check(ctx, load_library().dapq_recall(ctx, idx_gold.data_ptr(), idx_pred.data_ptr(), pl_p, kk_p, len(kk),
+                                           recall_out.data_ptr(), _stream(stream)))
 
 
 def dapq_evict(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, cu_rows, prompt_len, k_keep,

@@ -427,6 +427,22 @@ dapq_status dapq_compact_kv(dapq_ctx* ctx, const dapq_cache_view* cache, const i
   return DAPQ_OK;
 }
 
+dapq_status dapq_recall(dapq_ctx* ctx, const int32_t* idx_gold, const int32_t* idx_pred,
+                        const int32_t* prompt_len_host, const int32_t* k_keep_host, int32_t batch,
+                        float* recall_out, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!idx_gold || !idx_pred || !prompt_len_host || !k_keep_host || !recall_out)
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_recall: NULL argument");
+  SeqTable t;
+  dapq_status st = build_table(ctx, batch, nullptr, prompt_len_host, nullptr, k_keep_host, nullptr, &t);
+  if (st != DAPQ_OK) return st;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = launch_recall(idx_gold, idx_pred, t.cu_keep[batch], t, ctx->dims.n_kv_heads, recall_out,
+                                (cudaStream_t)stream, &ctx->log);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "recall kernel");
+  return DAPQ_OK;
+}
+
 dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
                        const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
                        float* scores_out, void* stream) {

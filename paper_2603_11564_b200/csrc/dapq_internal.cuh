@@ -64,7 +64,7 @@ __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
 
 // Kernel kinds, for launch accounting and the optional per-kernel event timing.
 enum KernelKind : int { kKindRope = 0, kKindSweep1, kKindLseMerge, kKindSweep2, kKindTopk, kKindCompact, kKindPool,
-                        kKindCount };
+                        kKindRecall, kKindCount };
 
 // Counts launches and, while profiling is on, brackets every launch with CUDA events on
 // the launching stream (implemented in api.cu; events come from a host-side pool).
@@ -114,6 +114,10 @@ cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx,
 // pooled[kvh, j] = max / mean of scores[kvh, j - kernel/2 .. j + kernel/2] within each sequence.
 cudaError_t launch_pool(const float* scores, float* pooled, int64_t stride, const SeqTable& t, int n_kv_heads,
                         int kernel, int mode, cudaStream_t s, LaunchLog* log);
+
+// recall[b, kvh] = |gold ∩ pred| / |gold| for two ascending index lists per (sequence, KV head).
+cudaError_t launch_recall(const int32_t* gold, const int32_t* pred, int64_t idx_stride, const SeqTable& t,
+                          int n_kv_heads, float* recall, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, int64_t idx_stride,
                            void* k_out, void* v_out, const SeqTable& t, int n_kv_heads, int* status,

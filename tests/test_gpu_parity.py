@@ -371,3 +371,28 @@ def test_pooled_selection_matches_oracle(dq, mode, kernel):
                 pooled = orc.pool_scores(s[h, cu_p[b]:cu_p[b + 1]].astype(np.float64), kernel, "max")
                 np.testing.assert_array_equal(idx[h, cu_k[b]:cu_k[b + 1]].cpu().numpy(), orc.topk_select(pooled, w.keep[b]))
     dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------------------------ recall (Section 3.3, Eq. 1-3)
+def test_recall_matches_oracle(dq):
+    rng = np.random.default_rng(12)
+    lens, keep = (900, 17, 5000), (64, 17, 1)
+    w = _small(lens=lens, keep=keep, n_q_heads=4, n_kv_heads=2, n_pseudo=4, n_needles=0, outlier_channels=0)
+    KT = int(w.cu_keep[-1])
+    gold = np.zeros((2, KT), dtype=np.int32)
+    pred = np.zeros((2, KT), dtype=np.int32)
+    for h in range(2):
+        for b, (L, K) in enumerate(zip(lens, keep)):
+            sl = slice(int(w.cu_keep[b]), int(w.cu_keep[b + 1]))
+            gold[h, sl] = np.sort(rng.choice(L, K, replace=False))
+            pred[h, sl] = np.sort(rng.choice(L, K, replace=False)) if (h + b) % 2 else gold[h, sl]
+    ctx = _ctx(dq, w)
+    out = torch.full((3, 2), -1.0, dtype=torch.float32, device="cuda")
+    dq.dapq_recall(ctx, torch.from_numpy(gold).cuda(), torch.from_numpy(pred).cuda(), lens, keep, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    for h in range(2):
+        for b in range(3):
+            sl = slice(int(w.cu_keep[b]), int(w.cu_keep[b + 1]))
+            assert got[b, h] == pytest.approx(orc.recall(gold[h, sl], pred[h, sl]), abs=1e-7), (b, h)
+    dq.dapq_destroy(ctx)
