@@ -14,6 +14,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 compact_kv_kernel(const CacheDev cv, int elem_bytes, const int32_t* __restrict__ idx, int64_t idx_stride,
                   uint4* __restrict__ k_out, uint4* __restrict__ v_out,
                   const __grid_constant__ SeqTable t, int* __restrict__ status) {
+  pdl_wait();
   const int kt = t.cu_keep[t.batch];
   const int64_t gid = (int64_t)blockIdx.x * kCompactThreads + threadIdx.x;
   const int r = (int)(gid / kPieces), piece = (int)(gid % kPieces);
@@ -46,13 +47,13 @@ cudaError_t launch_compact(int dtype, const CacheDev& cv, const int32_t* idx, in
   if (dtype == DAPQ_BF16) {
     constexpr int P = kHeadDim * 2 / 16;
     const dim3 grid((unsigned)(((int64_t)kt * P + kCompactThreads - 1) / kCompactThreads), n_kv_heads, 2);
-    compact_kv_kernel<P><<<grid, kCompactThreads, 0, s>>>(cv, 2, idx, idx_stride, (uint4*)k_out,
-                                                          (uint4*)v_out, t, status);
+    launch_pdl(compact_kv_kernel<P>, grid, dim3(kCompactThreads), 0, s, 1, cv, 2, idx, idx_stride, (uint4*)k_out,
+               (uint4*)v_out, t, status);
   } else {
     constexpr int P = kHeadDim * 4 / 16;
     const dim3 grid((unsigned)(((int64_t)kt * P + kCompactThreads - 1) / kCompactThreads), n_kv_heads, 2);
-    compact_kv_kernel<P><<<grid, kCompactThreads, 0, s>>>(cv, 4, idx, idx_stride, (uint4*)k_out,
-                                                          (uint4*)v_out, t, status);
+    launch_pdl(compact_kv_kernel<P>, grid, dim3(kCompactThreads), 0, s, 1, cv, 4, idx, idx_stride, (uint4*)k_out,
+               (uint4*)v_out, t, status);
   }
   log->end(s);
   return cudaGetLastError();

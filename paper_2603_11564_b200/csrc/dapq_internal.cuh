@@ -76,6 +76,43 @@ struct LaunchLog {
   void end(cudaStream_t s);
 };
 
+// ---- programmatic dependent launch --------------------------------------------------------
+// Every kernel of the eviction path is launched with programmatic stream serialization and
+// waits, before its first access to global memory, until the kernel before it has completed
+// and its writes are visible (pdl_wait): its launch is then prepared, and its CTAs' set-up done,
+// while the predecessor still runs.  The short kernels that precede a long one (rotation,
+// selection) also signal at their start that the next kernel may be scheduled (pdl_trigger); the
+// sweeps do not: their successors' CTAs would only sit on the SMs the next sweep needs (measured:
+// slower).  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with programmatic stream serialization (and a cluster of cluster_x CTAs if > 1).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, int cluster_x,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launchers (each returns the cudaError_t of its launch) -------------------------------
 // q_pre has element type `dtype`; q_rot is written as `out_mode`: bf16, fp32 (unrounded, for
 // the CUDA-core scorer) or a bf16 pair hi + lo with lo = bf16(q - hi) stored `lo_offset`

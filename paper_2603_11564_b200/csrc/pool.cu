@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kPoolThreads)
 pool_scores_kernel(const float* __restrict__ scores, float* __restrict__ pooled, int64_t stride,
                    const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable tiles, int kernel, int mode) {
   __shared__ float tile[kPoolTile + 2 * kMaxHalo];
+  pdl_wait();
   const int b = find_segment(tiles.cu_chunk, t.batch, blockIdx.x);
   const int L = t.prompt_len[b], r = kernel / 2;
   const int j0 = (blockIdx.x - tiles.cu_chunk[b]) * kPoolTile;          // first position of this tile
@@ -55,7 +56,7 @@ cudaError_t launch_pool(const float* scores, float* pooled, int64_t stride, cons
   tiles.cu_chunk[t.batch] = n;
   tiles.n_chunks = n;
   log->begin(kKindPool, s);
-  pool_scores_kernel<<<dim3(n, n_kv_heads), kPoolThreads, 0, s>>>(scores, pooled, stride, t, tiles, kernel, mode);
+  launch_pdl(pool_scores_kernel, dim3(n, n_kv_heads), dim3(kPoolThreads), 0, s, 1, scores, pooled, stride, t, tiles, kernel, mode);
   log->end(s);
   return cudaGetLastError();
 }

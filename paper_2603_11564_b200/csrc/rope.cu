@@ -32,6 +32,8 @@ __global__ void __launch_bounds__(kHeadDim / 2 * kHeadsPerBlock)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
                      int n_q_heads, int n_pseudo, int64_t lo_offset) {
+  pdl_trigger();
+  pdl_wait();
   const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const int h = blockIdx.z * kHeadsPerBlock + threadIdx.y;
   if (h >= n_q_heads) return;
@@ -61,17 +63,17 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
   dim3 grid(dm.n_pseudo, t.batch, (dm.n_q_heads + kHeadsPerBlock - 1) / kHeadsPerBlock);
   dim3 block(kHeadDim / 2, kHeadsPerBlock);
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
-    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true><<<grid, block, 0, s>>>(
-        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset);
+    launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
-    rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false><<<grid, block, 0, s>>>(
-        (const __nv_bfloat16*)q_pre, (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+    launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   } else if (dtype == DAPQ_BF16) {
-    rope_pseudo_q_kernel<__nv_bfloat16, float, false><<<grid, block, 0, s>>>(
-        (const __nv_bfloat16*)q_pre, (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+    launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, float, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
+               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   } else {
-    rope_pseudo_q_kernel<float, float, false><<<grid, block, 0, s>>>((const float*)q_pre, (float*)q_rot,
-                                                                     inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+    launch_pdl(rope_pseudo_q_kernel<float, float, false>, grid, block, 0, s, 1, (const float*)q_pre, (float*)q_rot,
+               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
   }
   log->end(s);
   return cudaGetLastError();

@@ -153,12 +153,13 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   if ((e = cudaFuncSetAttribute(score_sweep2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
   if (lse_in == nullptr) {
     log->begin(kKindSweep1, s);
-    score_sweep1_kernel<<<dim3(plan.ct1.n_chunks, dm.n_kv_heads), kThreads, kSmemBytes, s>>>(plan.tm_k1, plan.tm_q, t, plan.ct1, a);
+    launch_pdl(score_sweep1_kernel, dim3(plan.ct1.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k1,
+               plan.tm_q, t, plan.ct1, a);
     log->end(s);
   }
   log->begin(kKindSweep2, s);
-  score_sweep2_kernel<<<dim3(plan.ct2.n_chunks, dm.n_kv_heads), kThreads, kSmemBytes, s>>>(plan.tm_k2, plan.tm_q, t, plan.ct2,
-                                                                                       plan.ct1, a);
+  launch_pdl(score_sweep2_kernel, dim3(plan.ct2.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k2,
+             plan.tm_q, t, plan.ct2, plan.ct1, a);
   log->end(s);
   return cudaGetLastError();
 }

@@ -82,7 +82,8 @@ struct Bars {
   __device__ __forceinline__ uint32_t half_done(int i) const { return base + 8u * (12 + i); }
 };
 
-// Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync.
+// Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync, then
+// the wait for the kernel before this one (its set-up overlaps that kernel's tail).
 // Returns the tensor-memory base address.
 __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, int n_stages) {
   const int warp = threadIdx.x >> 5;
@@ -106,6 +107,7 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                                                   // global memory is touched only from here on
   return *reinterpret_cast<volatile uint32_t*>(smem + Smem::tmem_ptr);
 }
 

@@ -55,6 +55,8 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(smem_raw);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TopkSmem));   // [cache_keys]
 
+  pdl_trigger();
+  pdl_wait();
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int n_cta = (int)cluster.num_blocks();               // CTAs of this cluster (1, 2, 4 or 8)
@@ -226,20 +228,9 @@ cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx,
   cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)(sizeof(TopkSmem) + (size_t)kMaxSliceSmem * sizeof(uint32_t)));
   if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(t.batch * n_cta, n_kv_heads);
-  cfg.blockDim = dim3(kTopkThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = n_cta;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   log->begin(kKindTopk, s);
-  e = cudaLaunchKernelEx(&cfg, topk_select_kernel, scores, score_stride, idx, idx_stride, t, cache_keys);
+  e = launch_pdl(topk_select_kernel, dim3(t.batch * n_cta, n_kv_heads), dim3(kTopkThreads), smem, s, n_cta, scores,
+                 score_stride, idx, idx_stride, t, cache_keys);
   log->end(s);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
