@@ -34,13 +34,17 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
   }
   if (!kMasked || m_raw > -CUDART_INF_F) {
     const float neg = -m_raw * c;
-    float s0 = 0.f, s1 = 0.f;
+    // pairs of columns on the packed fp32 pipe; 2^x by MUFU or, for the pairs of kPolyPairMask, by polynomial
+    const float2 c2 = make_float2(c, c), neg2 = make_float2(neg, neg);
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int e = 0; e < 32; e += 2) {
-      s0 += ex2_sel(fmaf(x[e], c, neg), e);
-      s1 += ex2_sel(fmaf(x[e + 1], c, neg), e + 1);
+    for (int e = 0; e < 32; e += 4) {
+      const float2 x0 = __ffma2_rn(make_float2(x[e], x[e + 1]), c2, neg2);
+      const float2 x1 = __ffma2_rn(make_float2(x[e + 2], x[e + 3]), c2, neg2);
+      acc0 = __fadd2_rn(acc0, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
+      acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
     }
-    z += s0 + s1;
+    z += (acc0.x + acc0.y) + (acc1.x + acc1.y);
   }
 }
 

@@ -27,7 +27,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   if (nt <= 0) return;
   const Bars bars{sbase + Smem::bars};
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
-  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] base-2 lse of the resident query group
+  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
   const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages2);
 
   if (warp == 0) {
@@ -78,6 +78,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const int r = quad * 32 + lane;                             // accumulator row of this thread
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2e;
+    const float2 c2 = make_float2(c, c);
     int job = 0;
     bool ok = true;
     // (an aborting group still walks every query group: the other group waits for it at the barriers)
@@ -121,7 +122,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           }
           if (a.lse_out && chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
         }
-        lse_s[row] = l2;
+        lse_s[row] = -l2;                                         // negated: the epilogue adds it
       }
       epilogue_sync();
       // 32-column pieces of a job: group 0 takes the first h, group 1 the rest
@@ -133,7 +134,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = lane_addr + buf * 256;
-        float sum0 = 0.f, sum1 = 0.f;
+        float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
         uint32_t v[2][32];
         if (np > 0) tmem_ld32(taddr + p0 * 32, v[0]);
 #pragma unroll
@@ -144,22 +145,25 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             const int ch = p0 + k;
             const int valid = rows_g - ch * 32;                 // >= 32 except in the last piece
             if (valid >= 32) {
+              // pairs of columns on the packed fp32 pipe: x = s * c - lse, then 2^x by MUFU or polynomial
 #pragma unroll
               for (int e = 0; e < 32; e += 4) {
                 const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
-                sum0 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e]), c, -l4.x), e);
-                sum1 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 1]), c, -l4.y), e + 1);
-                sum0 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 2]), c, -l4.z), e + 2);
-                sum1 += ex2_sel(fmaf(__uint_as_float(v[k & 1][e + 3]), c, -l4.w), e + 3);
+                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[k & 1][e]), __uint_as_float(v[k & 1][e + 1])), c2,
+                                             make_float2(l4.x, l4.y));
+                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[k & 1][e + 2]), __uint_as_float(v[k & 1][e + 3])), c2,
+                                             make_float2(l4.z, l4.w));
+                acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
+                acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
               }
             } else {
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (e < valid) sum0 += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, -lse_s[ch * 32 + e]));
+                if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, lse_s[ch * 32 + e]));
             }
           }
         }
-        float sum = sum0 + sum1;
+        float sum = (acc.x + acc.y) + (acc1.x + acc1.y);
         const uint32_t xcol = taddr + h * 32;                   // a column group 1 has consumed (or nobody reads)
         if (eg == 1) {
           tmem_st1(xcol, __float_as_uint(sum));

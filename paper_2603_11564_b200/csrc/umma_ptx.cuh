@@ -129,25 +129,26 @@ __device__ __forceinline__ float ex2(float x) {
 // 1.5 * 2^23 trick, a degree-3 minimax polynomial for 2^f on [-0.5, 0.5] (relative error below
 // 7.5e-5), and n added into the exponent field.  Inputs below -125 give 2^-125.  The scorer's
 // epilogues owe one exponential per (query, key) pair and the MUFU pipe delivers only 16 per
-// clock and SM, so every kPolyEvery-th element of a piece takes this path.
-#ifndef DAPQ_POLY_EVERY
-#define DAPQ_POLY_EVERY 4
+// clock and SM, so a quarter of the column pairs of a piece takes this path.  Everything works
+// on two values at once with the packed fp32 instructions of sm_100 (one FFMA2 / FADD2 per
+// register pair): 2^x.x and 2^x.y on the MUFU, or both by the polynomial.
+#ifndef DAPQ_POLY_PAIR_MASK
+#define DAPQ_POLY_PAIR_MASK 0x8888u
 #endif
-constexpr int kPolyEvery = DAPQ_POLY_EVERY;
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -125.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.0551716648f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
-// The e-th element of a 32-column piece (e is a constant after unrolling): polynomial for
-// every kPolyEvery-th one, MUFU otherwise; kPolyEvery = 0 keeps everything on the MUFU.
-__device__ __forceinline__ float ex2_sel(float x, int e) {
-  if (kPolyEvery > 0 && (e % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery > 0 ? kPolyEvery : 1) - 1) return ex2_poly(x);
-  return ex2(x);
+constexpr uint32_t kPolyPairMask = DAPQ_POLY_PAIR_MASK;   // bit p: pair p of a 32-column piece takes the polynomial
+__device__ __forceinline__ float2 ex2_pair_mufu(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+__device__ __forceinline__ float2 ex2_pair_poly(float2 x) {
+  x.x = fmaxf(x.x, -125.f);
+  x.y = fmaxf(x.y, -125.f);
+  const float2 magic = make_float2(12582912.f, 12582912.f), neg_magic = make_float2(-12582912.f, -12582912.f);
+  const float2 t = __fadd2_rn(x, magic);
+  const float2 n = __fadd2_rn(t, neg_magic);
+  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(make_float2(0.0551716648f, 0.0551716648f), f, make_float2(0.2426111251f, 0.2426111251f));
+  p = __ffma2_rn(p, f, make_float2(0.6932609677f, 0.6932609677f));
+  p = __ffma2_rn(p, f, make_float2(0.9999280572f, 0.9999280572f));
+  return make_float2(__uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23)),
+                     __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23)));
 }
 
 // Three-input maximum (one instruction on sm_100).
