@@ -45,8 +45,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 NCU_TRAFFIC_BYTES = {
     # profiles/evict_kernels_llama3_8b_32k.md (a 2-layer run of the same command; traffic per launch does not
     # depend on the number of layers)
-    ("sweep1", "llama3_8b_32k"): 68345088 + 932608,
-    ("sweep2", "llama3_8b_32k"): 68804096 + 924160,
+    ("sweep1", "llama3_8b_32k"): 68345856 + 1063424,
+    ("sweep2", "llama3_8b_32k"): 68795392 + 1159680,
 }
 
 
@@ -293,6 +293,12 @@ def run_ours(args, w: gi.Workload):
         step()
     prof = dq.dapq_profile_read(ctx)
     dq.dapq_profile(ctx, False)
+    if sampler:
+        # short runs end before nvidia-smi has sampled a few times: keep the same load on for ~0.5 s
+        t_end = time.perf_counter() + 0.5
+        while time.perf_counter() < t_end:
+            step()
+            torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
 
     ms_total = max_over_ranks(ms_total, world, dev)
