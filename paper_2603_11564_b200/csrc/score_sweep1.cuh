@@ -5,29 +5,31 @@
 //   D[query, key] = Q_blk K_tile^T, queries on tensor-memory lanes, 192 keys per tile.
 // A job is one [128 queries x 192 keys] accumulator; the two query blocks of a group own one
 // accumulator each, so the MMAs of one block run while the other block's accumulator is read.
-// Both epilogue groups work on every job, 96 key columns each: thread (group g, row r) keeps
+// All four epilogue groups work on every job, 48 key columns each: thread (group g, row r) keeps
 // the statistics of query row r over the columns of its group, which become slot g of the
-// row's per-chunk partials.
+// row's per-chunk partials.  Sixteen epilogue warps (four per scheduler) hide the latency of
+// the tensor-memory loads and of the hand-offs, so each reads its columns in plain 16-column
+// pieces.
 #pragma once
 #include "score_umma_common.cuh"
 
 namespace dapq {
 namespace umma {
 
-// Running max / sum of exp over one 32-column piece of an accumulator row.
+// Running max / sum of exp over one 16-column piece of an accumulator row.
 // lim: last visible column of the piece's tile for this thread's pseudo query (masked tiles).
 template <bool kMasked>
 __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int lim, float c, float& m_raw, float& z) {
-  float x[32];
+  float x[16];
 #pragma unroll
-  for (int e = 0; e < 32; ++e) {
+  for (int e = 0; e < 16; ++e) {
     x[e] = __uint_as_float(v[e]);
     if (kMasked && col0 + e > lim) x[e] = -CUDART_INF_F;
   }
   float cmax = max3(x[0], x[1], x[2]);
 #pragma unroll
-  for (int e = 3; e < 31; e += 2) cmax = max3(cmax, x[e], x[e + 1]);
-  cmax = fmaxf(cmax, x[31]);
+  for (int e = 3; e < 15; e += 2) cmax = max3(cmax, x[e], x[e + 1]);
+  cmax = fmaxf(cmax, x[15]);
   if (cmax > m_raw) {
     z *= ex2((m_raw - cmax) * c);
     m_raw = cmax;
@@ -38,7 +40,7 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
     const float2 c2 = make_float2(c, c), neg2 = make_float2(neg, neg);
     float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int e = 0; e < 32; e += 4) {
+    for (int e = 0; e < 16; e += 4) {
       const float2 x0 = __ffma2_rn(make_float2(x[e], x[e + 1]), c2, neg2);
       const float2 x1 = __ffma2_rn(make_float2(x[e + 2], x[e + 3]), c2, neg2);
       acc0 = __fadd2_rn(acc0, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
@@ -48,17 +50,16 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
   }
 }
 
-// This group's 96 columns of one accumulator, in three pieces with the next piece's load in flight.
+// This group's 48 columns of one accumulator, in three 16-column pieces.
 __device__ __forceinline__ void row_stats_job(uint32_t taddr, int col0, bool masked, int lim, float c, float& m_raw,
                                               float& z) {
-  uint32_t v[2][32];
-  tmem_ld32(taddr, v[0]);
 #pragma unroll
-  for (int ch = 0; ch < 3; ++ch) {
-    tmem_ld_wait_for(v[ch & 1]);
-    if (ch + 1 < 3) tmem_ld32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);
-    if (masked) row_stats_piece<true>(v[ch & 1], col0 + ch * 32, lim, c, m_raw, z);
-    else row_stats_piece<false>(v[ch & 1], col0 + ch * 32, lim, c, m_raw, z);
+  for (int ch = 0; ch < kTile1 / kEpiGroups / 16; ++ch) {
+    uint32_t v[16];
+    tmem_ld16(taddr + ch * 16, v);
+    tmem_ld_wait_for16(v);
+    if (masked) row_stats_piece<true>(v, col0 + ch * 16, lim, c, m_raw, z);
+    else row_stats_piece<false>(v, col0 + ch * 16, lim, c, m_raw, z);
   }
 }
 
@@ -130,12 +131,12 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
   } else {
     // ============================================================================== epilogue
-    const int eg = (warp - 2) >> 2;                             // epilogue group 0 / 1: key columns 96 eg .. 96 eg + 95
+    const int eg = (warp - 2) >> 2;                             // epilogue group 0 .. 3: key columns 48 eg .. 48 eg + 47
     const int quad = warp & 3;                                  // TMEM lane quadrant of this warp
     const int r = quad * 32 + lane;                             // accumulator row of this thread
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2e;
-    const int col0 = eg * (kTile1 / 2);
+    const int col0 = eg * (kTile1 / kEpiGroups);
     uint32_t use0 = 0u, use1 = 0u;                              // jobs taken from each accumulator
     bool ok = true;
     for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
@@ -164,7 +165,7 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
       }
       // partials: slot eg of this thread's rows
-      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * 2 + eg) * (a.n_qgroups * kGroupRows) +
+      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * kEpiGroups + eg) * (a.n_qgroups * kGroupRows) +
                       qg * kGroupRows;
       if (qg * kGroupRows + r < a.rows_total) pbase[r] = make_float2(m_raw0 * c, z0);
       if (mb == 2 && qg * kGroupRows + 128 + r < a.rows_total) pbase[128 + r] = make_float2(m_raw1 * c, z1);

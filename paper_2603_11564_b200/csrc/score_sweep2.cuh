@@ -2,11 +2,13 @@
 // summed over the N pseudo queries and the G query heads of the KV head's group.
 //
 //   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
-// A job is one [128 keys x 256 queries] accumulator (two fit).  Both epilogue groups work on
-// every job, half of the query columns each; group 1 hands its partial sum to group 0 through
-// a consumed column of the same accumulator, and group 0's thread (lane = key) stores the
-// key's score: one coalesced fp32 per lane.  Before the first job the epilogue threads merge
-// the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the resident query rows.
+// A job is one [128 keys x 256 queries] accumulator (two fit).  All four epilogue groups work
+// on every job, a quarter of the query columns each (sixteen epilogue warps, four per scheduler,
+// hide the latency of the tensor-memory loads and of the hand-offs); groups 1-3 hand their
+// partial sums to group 0 through consumed columns of the same accumulator, and group 0's thread
+// (lane = key) stores the key's score: one coalesced fp32 per lane.  Before the first job the
+// epilogue threads merge the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the
+// resident query rows.
 #pragma once
 #include "score_umma_common.cuh"
 
@@ -87,7 +89,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk
       // partials of row eg*128 + r in a fixed order, or converts the caller's value
       if (qg > 0) epilogue_sync();                              // the previous group's values are no longer read
-      {
+      if (eg < 2) {
         const int row = eg * 128 + r, grow = qg * kGroupRows + row;
         float l2 = 0.f;
         if (grow < a.rows_total) {
@@ -95,18 +97,19 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
           } else {
             const int rows_pad = a.n_qgroups * kGroupRows;
-            const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * 2 * rows_pad + grow;
-            const int64_t step = (int64_t)a.n_kv_heads * 2 * rows_pad;
+            const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * kEpiGroups * rows_pad + grow;
+            const int64_t step = (int64_t)a.n_kv_heads * kEpiGroups * rows_pad;
             const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
             // one pass, eight independent loads in flight; (max, sum) merged in chunk order
             float mx = -CUDART_INF_F, z = 0.f;
-            for (int c0 = 0; c0 < nc; c0 += 4) {
+            for (int c0 = 0; c0 < nc; c0 += 2) {
               float2 q[8];
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
+              for (int u = 0; u < 2; ++u) {
                 const bool in = c0 + u < nc;
-                q[2 * u] = in ? __ldg(p + (c0 + u) * step) : make_float2(-CUDART_INF_F, 0.f);
-                q[2 * u + 1] = in ? __ldg(p + (c0 + u) * step + rows_pad) : make_float2(-CUDART_INF_F, 0.f);
+#pragma unroll
+                for (int g = 0; g < kEpiGroups; ++g)
+                  q[kEpiGroups * u + g] = in ? __ldg(p + (c0 + u) * step + g * rows_pad) : make_float2(-CUDART_INF_F, 0.f);
               }
               float m8 = q[0].x;
 #pragma unroll
@@ -125,9 +128,9 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         lse_s[row] = -l2;                                         // negated: the epilogue adds it
       }
       epilogue_sync();
-      // 32-column pieces of a job: group 0 takes the first h, group 1 the rest
-      const int nch = (rows_g + 31) >> 5, h = (nch + 1) >> 1;
-      const int p0 = eg ? h : 0, np = eg ? nch - h : h;
+      // 32-column pieces of a job: group g takes pieces [g nch / 4, (g + 1) nch / 4)
+      const int nch = (rows_g + 31) >> 5;
+      const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
       for (int ti = 0; ti < nt && ok; ++ti, ++job) {
         const int buf = job & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), (job >> 1) & 1, abort_flag, a.status));
@@ -135,13 +138,12 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tc_fence_after();
         const uint32_t taddr = lane_addr + buf * 256;
         float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-        uint32_t v[2][32];
-        if (np > 0) tmem_ld32(taddr + p0 * 32, v[0]);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 2; ++k) {
           if (k < np) {
-            tmem_ld_wait_for(v[k & 1]);
-            if (k + 1 < np) tmem_ld32(taddr + (p0 + k + 1) * 32, v[(k + 1) & 1]);
+            uint32_t v[32];
+            tmem_ld32(taddr + (p0 + k) * 32, v);
+            tmem_ld_wait_for(v);
             const int ch = p0 + k;
             const int valid = rows_g - ch * 32;                 // >= 32 except in the last piece
             if (valid >= 32) {
@@ -149,9 +151,9 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
               for (int e = 0; e < 32; e += 4) {
                 const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
-                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[k & 1][e]), __uint_as_float(v[k & 1][e + 1])), c2,
+                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2,
                                              make_float2(l4.x, l4.y));
-                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[k & 1][e + 2]), __uint_as_float(v[k & 1][e + 3])), c2,
+                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2,
                                              make_float2(l4.z, l4.w));
                 acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
                 acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
@@ -159,15 +161,18 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             } else {
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[k & 1][e]), c, lse_s[ch * 32 + e]));
+                if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[e]), c, lse_s[ch * 32 + e]));
             }
           }
         }
         float sum = (acc.x + acc.y) + (acc1.x + acc1.y);
-        const uint32_t xcol = taddr + h * 32;                   // a column group 1 has consumed (or nobody reads)
-        if (eg == 1) {
-          tmem_st1(xcol, __float_as_uint(sum));
-          tmem_st_wait();
+        if (eg > 0) {
+          // hand the partial sum over in the first column this group has consumed (nothing to hand over
+          // if it had no columns), then release the accumulator
+          if (np > 0) {
+            tmem_st1(taddr + p0 * 32, __float_as_uint(sum));
+            tmem_st_wait();
+          }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) { mbar_arrive(bars.half_done(buf)); mbar_arrive(bars.acc_empty(buf)); }
@@ -175,7 +180,11 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job >> 1) & 1, abort_flag, a.status));
           if (!ok) break;
           tc_fence_after();
-          sum += __uint_as_float(tmem_ld1(xcol));
+#pragma unroll
+          for (int g = 1; g < kEpiGroups; ++g) {
+            const int gp0 = (g * nch) / kEpiGroups, gnp = ((g + 1) * nch) / kEpiGroups - gp0;
+            if (gnp > 0) sum += __uint_as_float(tmem_ld1(taddr + gp0 * 32));
+          }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.acc_empty(buf));

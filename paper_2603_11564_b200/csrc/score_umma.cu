@@ -21,13 +21,13 @@
 // 77 cycles whatever its size, so MMAs are made wide (N = 192 / 256: 105 / 139 cycles for
 // 128 x N x 16) and their descriptors cost one add each; a commit -> wait -> release -> issue
 // hand-off of an accumulator takes about 700 cycles, so a job is a whole [128 x 192 / 256]
-// block of 16 MMAs and both epilogue groups split the columns of every job, which halves the
-// time an accumulator is held.
+// block of 16 MMAs and all epilogue groups split the columns of every job, which shortens the
+// time an accumulator is held; four epilogue warps per scheduler hide the ~370-cycle latency
+// of a tensor-memory load and the hand-off waits behind each other's exponentials.
 //
-// CTA = (chunk of K tiles, KV head); 10 warps: warp 0 issues the TMA loads (query group, K
-// ring), warp 1 issues the MMAs and owns tensor memory, warps 2-9 are two epilogue groups
-// (4 warps = 128 TMEM lanes each) that read accumulators in 32-column pieces with the next
-// piece's load in flight.  Every mbarrier wait is bounded: after ~1 s the CTA raises the
+// CTA = (chunk of K tiles, KV head); 18 warps: warp 0 issues the TMA loads (query group, K
+// ring), warp 1 issues the MMAs and owns tensor memory, warps 2-17 are four epilogue groups
+// (4 warps = 128 TMEM lanes each) that split the columns of every accumulator.  Every mbarrier wait is bounded: after ~1 s the CTA raises the
 // timeout status, drains and returns normally.
 #include "score_sweep1.cuh"
 #include "score_sweep2.cuh"
@@ -106,7 +106,7 @@ bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int n_kv_head
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo) {
   const int rows_total = n_q_heads / n_kv_heads * n_pseudo;
   const int rows_pad = (rows_total + kGroupRows - 1) / kGroupRows * kGroupRows;
-  return (int64_t)(max_batch + kUmmaMaxChunks) * n_kv_heads * 2 * rows_pad;
+  return (int64_t)(max_batch + kUmmaMaxChunks) * n_kv_heads * kEpiGroups * rows_pad;
 }
 
 bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheDev& cv, const SeqTable& t,

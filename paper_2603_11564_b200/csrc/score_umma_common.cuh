@@ -12,7 +12,8 @@ constexpr int kTile2 = 128;                    // keys per K tile of sweep 2 (= 
 constexpr int kGroupRows = 256;                // query rows resident per group (2 blocks of 128)
 constexpr int kHalfBytesQ = kGroupRows * 128;  // one 64-channel half of a query group (32 KB)
 constexpr int kQBytes = 2 * kHalfBytesQ;       // 64 KB per precision part (hi / lo)
-constexpr int kThreads = 320;
+constexpr int kEpiGroups = 4;                  // epilogue groups of 4 warps (128 TMEM lanes each)
+constexpr int kThreads = 64 + kEpiGroups * 128;
 constexpr int kTmemCols = 512;
 
 // Shared memory of both sweeps (offsets from the 1024-aligned base): the query group as a
@@ -42,7 +43,7 @@ struct UmmaArgs {
   int32_t has_lo;            // the query operand carries a low-order bf16 part
   int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
   float scale_log2e;
-  float2* part;              // [n_chunks1, H_kv, 2, n_qgroups * 256] (running max, sum) in base 2
+  float2* part;              // [n_chunks1, H_kv, 4, n_qgroups * 256] (running max, sum) in base 2, one slot per group
   const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
   float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
   float* scores;
@@ -91,8 +92,8 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
     for (int s = 0; s < n_stages; ++s) { mbar_init(bars.k_full(s), 1); mbar_init(bars.k_empty(s), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bars.acc_full(i), 1);
-      mbar_init(bars.acc_empty(i), 8);      // all 8 epilogue warps read every accumulator
-      mbar_init(bars.half_done(i), 4);
+      mbar_init(bars.acc_empty(i), 4 * kEpiGroups);        // every epilogue warp reads every accumulator
+      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the groups that hand their partial sums to group 0
     }
     mbar_init(bars.q_full(), 1);
     mbar_init(bars.q_empty(), 1);
