@@ -180,11 +180,15 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job >> 1) & 1, abort_flag, a.status));
           if (!ok) break;
           tc_fence_after();
+          // the three partial sums: loads issued together, one wait (a group without columns left nothing)
+          uint32_t part[kEpiGroups - 1] = {0u, 0u, 0u};
 #pragma unroll
           for (int g = 1; g < kEpiGroups; ++g) {
             const int gp0 = (g * nch) / kEpiGroups, gnp = ((g + 1) * nch) / kEpiGroups - gp0;
-            if (gnp > 0) sum += __uint_as_float(tmem_ld1(taddr + gp0 * 32));
+            if (gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g - 1]);
           }
+          tmem_ld_wait3(part[0], part[1], part[2]);
+          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + __uint_as_float(part[2]);
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.acc_empty(buf));
