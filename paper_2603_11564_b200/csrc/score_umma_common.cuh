@@ -129,6 +129,17 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
                                              volatile int* abort_flag) {
   int li = 0;                                               // K tiles loaded so far
   bool ok = true;
+  auto load_tile = [&](int ti) {
+    const int s = li % kStages;
+    mbar_expect_tx(bars.k_full(s), kStage);
+    const int row = w.row_base + (w.t0 + ti) * kTile;
+    tma_load_3d(sbase + Smem::k + s * kStage, tm_k, bars.k_full(s), 0, row, kvh);
+    tma_load_3d(sbase + Smem::k + s * kStage + kHalf, tm_k, bars.k_full(s), 64, row, kvh);
+    ++li;
+  };
+  // The first K tiles go out before the queries: they come from further away (DRAM in sweep 1).
+  const int n_first = min(kStages, w.nt);
+  for (int ti = 0; ti < n_first; ++ti) load_tile(ti);
   for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
     const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
     const int mb = (rows_g + 127) / 128;
@@ -141,14 +152,11 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
         for (int m = 0; m < mb; ++m)
           tma_load_2d(sbase + (part ? Smem::q_lo : Smem::q_hi) + half * kHalfBytesQ + m * 128 * 128, tm_q, bars.q_full(),
                       half * 64, part * a.lo_row_offset + w.qrow_base + qg * kGroupRows + m * 128);
-    for (int ti = 0; ti < w.nt; ++ti, ++li) {
+    for (int ti = (qg == 0 ? n_first : 0); ti < w.nt; ++ti) {
       const int s = li % kStages;
       if (li >= kStages) ok = mbar_wait(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status);
       if (!ok) break;
-      mbar_expect_tx(bars.k_full(s), kStage);
-      const int row = w.row_base + (w.t0 + ti) * kTile;
-      tma_load_3d(sbase + Smem::k + s * kStage, tm_k, bars.k_full(s), 0, row, kvh);
-      tma_load_3d(sbase + Smem::k + s * kStage + kHalf, tm_k, bars.k_full(s), 64, row, kvh);
+      load_tile(ti);
     }
   }
   if (!ok) {
