@@ -185,12 +185,13 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
           prompt_len: Sequence[int], k_keep: Sequence[int], rope_base: float,
           scale: Optional[float] = None,
           pos_start: Optional[Sequence[int]] = None, pool_mode: str = "none",
-          pool_kernel: int = 1) -> Dict[str, object]:
+          pool_kernel: int = 1, inv_freq: Optional[np.ndarray] = None) -> Dict[str, object]:
     """The whole path for one layer (Figure 1): rotate, score, select, compact.
 
     q_pre [B, H_q, N, d] pre-RoPE pseudo queries (any float dtype; converted exactly
     to float64); k, v [H_kv, R, d] packed cache whose sequence b owns rows
     cu_rows[b] .. cu_rows[b+1] (L_b prompt rows, then N synthetic rows).
+    inv_freq [d/2] replaces the frequencies base^(-2c/d) (models with scaled RoPE).
     With pool_mode "max" / "avg" the selection runs on the pooled scores (returned as
     "pooled"); "scores" are always the unpooled Eq. 4 sums.
     Returns per-sequence lists: scores [H_kv, L_b], idx [H_kv, K_b] (sequence-local),
@@ -207,7 +208,7 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
         r0 = int(cu_rows[b])
         assert int(cu_rows[b + 1]) - r0 == L + n
         p0 = L if pos_start is None else int(pos_start[b])
-        q_rot = rope_pseudo_q(np.asarray(q_pre[b], dtype=np.float64), p0, rope_base)
+        q_rot = rope_pseudo_q(np.asarray(q_pre[b], dtype=np.float64), p0, rope_base, inv_freq)
         k_seq = k[:, r0:r0 + L + n]
         v_seq = v[:, r0:r0 + L + n]
         res = score_sequence(q_rot, k_seq, L, G, scale)

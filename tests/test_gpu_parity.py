@@ -396,3 +396,41 @@ def test_recall_matches_oracle(dq):
             sl = slice(int(w.cu_keep[b]), int(w.cu_keep[b + 1]))
             assert got[b, h] == pytest.approx(orc.recall(gold[h, sl], pred[h, sl]), abs=1e-7), (b, h)
     dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------- caller-supplied RoPE frequencies, shifted positions
+def test_evict_with_scaled_rope_frequencies(dq):
+    """Frequencies of a scaled-RoPE model (long wavelengths divided by 8, as Llama-3.1 does) go in
+    through inv_freq; the oracle rotates with the same table."""
+    w = _small(lens=(900, 333), keep=(50, 20), n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    inv = orc.rope_inv_freq(128, w.rope_base)
+    inv = np.where(2 * np.pi / inv > 8192, inv / 8.0, inv)
+    data = gi.draw_layer(w, 0, "cpu")
+    ref = orc.evict(util.to_f64(data["q_pre"]), util.to_f64(data["k"]), util.to_f64(data["v"]), w.cu_rows,
+                    w.prompt_lens, w.keep, w.rope_base, inv_freq=inv)
+    plain = util.oracle_evict(w, data)
+    assert not np.allclose(ref["scores"][0], plain["scores"][0], rtol=1e-3)       # the table matters
+    ctx = _ctx(dq, w, inv_freq=list(inv))
+    _check_evict(w, data, _gpu_evict(dq, w, data, ctx), ref)
+    dq.dapq_destroy(ctx)
+
+
+def test_shifted_positions_through_rope_and_score(dq):
+    """The paper's position ablation (Section 6.3: pseudo queries placed at L_p + offset) through the
+    separate entry points: dapq_rope_pseudo_q with pos_start = L_b + offset, then dapq_score."""
+    w = _small(lens=(700,), keep=(1,), n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    offset = 4096
+    ctx = _ctx(dq, w)
+    q_rot = torch.empty_like(data["q_pre"]).cuda()
+    dq.dapq_rope_pseudo_q(ctx, data["q_pre"].cuda(), [700 + offset], q_rot)
+    scores = torch.empty((2, 700), dtype=torch.float32, device="cuda")
+    dq.dapq_score(ctx, q_rot, data["k"].cuda(), w.cu_rows, w.prompt_lens, scores)
+    dq.dapq_poll_status(ctx)
+    # both sides score the rotated queries as stored (bf16)
+    q_ref = util.to_f64(q_rot[0])
+    ref = orc.score_sequence(q_ref, util.to_f64(data["k"]), 700, w.group)["scores"]
+    util.assert_scores_close(scores.cpu().double().numpy(), ref, "shifted positions")
+    want = orc.rope_pseudo_q(util.to_f64(data["q_pre"][0]), 700 + offset, w.rope_base)
+    assert np.all(np.abs(q_ref - want) <= 2.0 ** -8 * np.abs(want) + 1e-7)
+    dq.dapq_destroy(ctx)
