@@ -75,7 +75,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
   } else {
     // ============================================================================== epilogue
-    const int eg = (warp - 2) >> 2;                             // epilogue group 0 / 1
+    const int eg = (warp - 2) >> 2;                             // epilogue group 0 .. 3
     const int quad = warp & 3;                                  // TMEM lane quadrant of this warp
     const int r = quad * 32 + lane;                             // accumulator row of this thread
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -83,7 +83,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const float2 c2 = make_float2(c, c);
     int job = 0;
     bool ok = true;
-    // (an aborting group still walks every query group: the other group waits for it at the barriers)
+    // (an aborting group still walks every query group: the other groups wait for it at the barriers)
     for (int qg = 0; qg < a.n_qgroups; ++qg) {
       const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
       // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk

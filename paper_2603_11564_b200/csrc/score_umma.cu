@@ -27,8 +27,9 @@
 //
 // CTA = (chunk of K tiles, KV head); 18 warps: warp 0 issues the TMA loads (query group, K
 // ring), warp 1 issues the MMAs and owns tensor memory, warps 2-17 are four epilogue groups
-// (4 warps = 128 TMEM lanes each) that split the columns of every accumulator.  Every mbarrier wait is bounded: after ~1 s the CTA raises the
-// timeout status, drains and returns normally.
+// (4 warps = 128 TMEM lanes each) that split the columns of every accumulator.  Every
+// mbarrier wait is bounded: after ~1 s the CTA raises the timeout status, drains and returns
+// normally.
 #include "score_sweep1.cuh"
 #include "score_sweep2.cuh"
 
