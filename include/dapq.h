@@ -15,7 +15,7 @@
  *   3. dapq_topk_select    M_retain = TopK_j S(j)                       (Section 4.2, Eq. 5)
  *   4. dapq_compact_kv     keep the K/V rows in M_retain, drop the rest and every
  *                          synthetic token (Section 4.2, last paragraph; Figure 1).
- *   5. dapq_evict          1-4 for one layer's cache on one stream.
+ *   5. dapq_evict          1-4 for one layer's cache on one stream (dapq_evict_layers: every layer).
  *
  * Conventions
  *   - One process drives one GPU.  All kernels are asynchronous on the caller's
@@ -188,6 +188,20 @@ DAPQ_API dapq_status dapq_recall(dapq_ctx* ctx, const int32_t* idx_gold, const i
 DAPQ_API dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
                        const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
                        float* scores_out, void* stream);
+
+/* dapq_evict for every layer of a model, in layer order on one stream, with a budget per layer
+ * (Section 4.2 is applied to each layer's cache on its own; the paper keeps one budget for all
+ * layers, the layer-wise budgets of the PyramidKV baseline in Section 5.1 are the general case).
+ * q_pre, caches, k_out, v_out, idx_out: HOST arrays of n_layers entries holding what dapq_evict
+ * takes for one layer (idx_out, or any entry of it, may be NULL).  k_keep_host: host
+ * [n_layers, batch] when k_keep_layer_stride = batch, or one row shared by all layers when
+ * k_keep_layer_stride = 0.  Every layer uses the same workspace, so the layers run back to back;
+ * only launches are issued (no copies, no synchronisation), which makes the whole call
+ * capturable into a CUDA graph.  Stops at the first layer that fails and returns its status. */
+DAPQ_API dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre,
+                              const dapq_cache_view* caches, const int32_t* k_keep_host,
+                              int64_t k_keep_layer_stride, void* const* k_out, void* const* v_out,
+                              int32_t* const* idx_out, void* stream);
 
 /* dapq_evict for callers whose tensors live in host memory: q_pre, the cache view's k / v
  * and k_out / v_out / idx_out are HOST pointers (pinned memory gives full copy speed).

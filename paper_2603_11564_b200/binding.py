@@ -27,7 +27,7 @@ _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORT
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
            "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
-           "dapq_compact_kv", "dapq_evict", "dapq_evict_host", "dapq_score_static", "dapq_recall")
+           "dapq_compact_kv", "dapq_evict", "dapq_evict_layers", "dapq_evict_host", "dapq_score_static", "dapq_recall")
 
 
 class DapqError(RuntimeError):
@@ -88,6 +88,9 @@ def load_library() -> C.CDLL:
     lib.dapq_compact_kv.restype = C.c_int
     lib.dapq_evict.argtypes = [vp, vp, C.POINTER(dapq_cache_view), i32p, vp, vp, vp, f32p, vp]
     lib.dapq_evict.restype = C.c_int
+    lib.dapq_evict_layers.argtypes = [vp, C.c_int32, C.POINTER(vp), C.POINTER(dapq_cache_view), i32p, C.c_int64,
+                                      C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
+    lib.dapq_evict_layers.restype = C.c_int
     lib.dapq_evict_host.argtypes = [vp, vp, C.POINTER(dapq_cache_view), i32p, vp, vp, vp, vp]
     lib.dapq_evict_host.restype = C.c_int
     lib.dapq_recall.argtypes = [vp, vp, vp, i32p, i32p, C.c_int32, f32p, vp]
@@ -233,6 +236,27 @@ def dapq_evict(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, cu_ro
     kk, kk_p = _i32(k_keep)
     _check(ctx, load_library().dapq_evict(ctx, q_pre.data_ptr(), C.byref(view), kk_p, k_out.data_ptr(),
                                           v_out.data_ptr(), _ptr(idx_out), _ptr(scores_out), _stream(stream)))
+
+
+def dapq_evict_layers(ctx, q_pre: Sequence[torch.Tensor], k: Sequence[torch.Tensor], v: Sequence[torch.Tensor], cu_rows,
+                      prompt_len, k_keep, k_out: Sequence[torch.Tensor], v_out: Sequence[torch.Tensor],
+                      idx_out: Optional[Sequence[torch.Tensor]] = None, stream=None) -> None:
+    """k_keep: one budget row [batch] for all layers, or one row per layer [n_layers][batch]."""
+    n = len(k)
+    views = (dapq_cache_view * n)()
+    keep_alive = []
+    for l in range(n):
+        view = _view(k[l], v[l], cu_rows, prompt_len)
+        keep_alive.append(view)
+        C.memmove(C.byref(views, l * C.sizeof(dapq_cache_view)), C.byref(view), C.sizeof(dapq_cache_view))
+    budgets = np.asarray(k_keep, dtype=np.int32)
+    assert budgets.ndim == 1 or (budgets.ndim == 2 and budgets.shape[0] == n)
+    kk, kk_p = _i32(budgets.reshape(-1))
+    stride = budgets.shape[1] if budgets.ndim == 2 else 0
+    arr = lambda ts: (C.c_void_p * n)(*[t.data_ptr() for t in ts])
+    idx_arr = arr(idx_out) if idx_out is not None else None
+    _check(ctx, load_library().dapq_evict_layers(ctx, n, arr(q_pre), views, kk_p, stride, arr(k_out), arr(v_out),
+                                                 idx_arr, _stream(stream)))
 
 
 def dapq_evict_host(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, cu_rows, prompt_len, k_keep,

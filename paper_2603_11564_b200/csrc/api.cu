@@ -483,6 +483,22 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   return DAPQ_OK;
 }
 
+dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre,
+                              const dapq_cache_view* caches, const int32_t* k_keep_host,
+                              int64_t k_keep_layer_stride, void* const* k_out, void* const* v_out,
+                              int32_t* const* idx_out, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (n_layers < 0 || k_keep_layer_stride < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers: negative count or stride");
+  if (n_layers > 0 && (!q_pre || !caches || !k_keep_host || !k_out || !v_out))
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers: NULL argument");
+  for (int32_t l = 0; l < n_layers; ++l) {
+    const dapq_status st = dapq_evict(ctx, q_pre[l], &caches[l], k_keep_host + (int64_t)l * k_keep_layer_stride, k_out[l],
+                                      v_out[l], idx_out ? idx_out[l] : nullptr, nullptr, stream);
+    if (st != DAPQ_OK) return st;
+  }
+  return DAPQ_OK;
+}
+
 dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
                             const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
                             int32_t* idx_out_host, void* stream) {

@@ -434,3 +434,71 @@ def test_shifted_positions_through_rope_and_score(dq):
     want = orc.rope_pseudo_q(util.to_f64(data["q_pre"][0]), 700 + offset, w.rope_base)
     assert np.all(np.abs(q_ref - want) <= 2.0 ** -8 * np.abs(want) + 1e-7)
     dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------------------- every layer in one call, budgets per layer
+def _layer_cases(n_layers, lens, budgets, **kw):
+    ws = [_small(lens=lens, keep=budgets[l], **kw) for l in range(n_layers)]
+    return ws, [gi.draw_layer(ws[l], l, "cpu") for l in range(n_layers)]
+
+
+def _layer_buffers(ws, datas):
+    dev = "cuda"
+    q, k, v = ([d[x].to(dev) for d in datas] for x in ("q_pre", "k", "v"))
+    ko = [torch.empty((w.n_kv_heads, int(w.cu_keep[-1]), w.head_dim), dtype=k[0].dtype, device=dev) for w in ws]
+    vo = [torch.empty_like(t) for t in ko]
+    idx = [torch.empty((w.n_kv_heads, int(w.cu_keep[-1])), dtype=torch.int32, device=dev) for w in ws]
+    return q, k, v, ko, vo, idx
+
+
+def test_evict_layers_with_per_layer_budgets(dq):
+    """dapq_evict_layers with a budget row per layer (layer-wise budgets as in the PyramidKV baseline of
+    Section 5.1): every layer equals its own dapq_evict call bit for bit and the oracle's retained set."""
+    lens, budgets = (600, 210), [(60, 21), (120, 40), (17, 3)]
+    ws, datas = _layer_cases(3, lens, budgets, n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    q, k, v, ko, vo, idx = _layer_buffers(ws, datas)
+    ctx = _ctx(dq, ws[0])
+    dq.dapq_evict_layers(ctx, q, k, v, ws[0].cu_rows, ws[0].prompt_lens, budgets, ko, vo, idx)
+    dq.dapq_poll_status(ctx)
+    for l, (w, data) in enumerate(zip(ws, datas)):
+        one = _gpu_evict(dq, w, data, ctx)
+        assert np.array_equal(idx[l].cpu().numpy(), one["idx"]), f"layer {l}"
+        assert torch.equal(ko[l].cpu(), one["k_out"]) and torch.equal(vo[l].cpu(), one["v_out"]), f"layer {l}"
+        _check_evict(w, data, one, util.oracle_evict(w, data))
+    # one budget row shared by all layers
+    ws1, datas1 = _layer_cases(2, lens, [budgets[0]] * 2, n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    q, k, v, ko, vo, idx = _layer_buffers(ws1, datas1)
+    dq.dapq_evict_layers(ctx, q, k, v, ws1[0].cu_rows, ws1[0].prompt_lens, budgets[0], ko, vo, idx)
+    dq.dapq_poll_status(ctx)
+    for l, (w, data) in enumerate(zip(ws1, datas1)):
+        assert np.array_equal(idx[l].cpu().numpy(), _gpu_evict(dq, w, data, ctx)["idx"]), f"shared budgets, layer {l}"
+    dq.dapq_destroy(ctx)
+
+
+def test_evict_layers_replays_from_a_cuda_graph(dq):
+    """The multi-layer call only issues launches, so it can be captured once and replayed on new cache
+    contents: the replay equals an eager call on the same contents."""
+    lens, budgets = (500, 1300), [(50, 130)] * 3
+    ws, datas = _layer_cases(3, lens, budgets, n_needles=0)
+    q, k, v, ko, vo, idx = _layer_buffers(ws, datas)
+    ctx = _ctx(dq, ws[0])
+    args = (ws[0].cu_rows, ws[0].prompt_lens, budgets[0])
+    dq.dapq_evict_layers(ctx, q, k, v, *args, ko, vo, idx)                  # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        dq.dapq_evict_layers(ctx, q, k, v, *args, ko, vo, idx)
+    # new contents in the captured buffers: the layers of another draw
+    fresh = [gi.draw_layer(ws[l], l + 7, "cpu") for l in range(3)]
+    for l in range(3):
+        for dst, name in ((q, "q_pre"), (k, "k"), (v, "v")):
+            dst[l].copy_(fresh[l][name])
+        ko[l].zero_(); vo[l].zero_(); idx[l].zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    dq.dapq_poll_status(ctx)
+    for l in range(3):
+        one = _gpu_evict(dq, ws[l], fresh[l], ctx)
+        assert np.array_equal(idx[l].cpu().numpy(), one["idx"]), f"layer {l}"
+        assert torch.equal(ko[l].cpu(), one["k_out"]) and torch.equal(vo[l].cpu(), one["v_out"]), f"layer {l}"
+    dq.dapq_destroy(ctx)
