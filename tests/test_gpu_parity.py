@@ -502,3 +502,37 @@ def test_evict_layers_replays_from_a_cuda_graph(dq):
         assert np.array_equal(idx[l].cpu().numpy(), one["idx"]), f"layer {l}"
         assert torch.equal(ko[l].cpu(), one["k_out"]) and torch.equal(vo[l].cpu(), one["v_out"]), f"layer {l}"
     dq.dapq_destroy(ctx)
+
+
+# --------------------------------------------------- observation window taken from the prompt itself
+def test_prompt_window_variant_uses_the_same_entry_points(dq):
+    """The SnapKV-style window of Section 5.1's baselines (queries = the last N prompt tokens, query i sees
+    keys up to its own position, window rows always kept) is the same computation with prompt_len = L - N:
+    the window's rows play the part of the synthetic rows.  Reference: the causal attention matrix written
+    out with torch in float64."""
+    L, N, hq, hkv, keep = 1500, 32, 8, 2, 200
+    w = _small(lens=(L - N,), keep=(keep - N,), n_q_heads=hq, n_kv_heads=hkv, n_pseudo=N, n_needles=0)
+    data = gi.draw_layer(w, 0, "cpu")                            # k: [H_kv, L, d]; q_pre stands for the window's rotated queries
+    q_win, k = data["q_pre"], data["k"]
+    assert k.shape[1] == L
+    qd, kd = q_win[0].double(), k.double()
+    pos_q = torch.arange(L - N, L).view(N, 1)
+    visible = torch.arange(L).view(1, L) <= pos_q                 # causal: key j <= position of window query i
+    ref = torch.zeros(hkv, L - N, dtype=torch.float64)
+    for h in range(hq):
+        logits = (qd[h] @ kd[h // (hq // hkv)].T) / np.sqrt(128.0)
+        probs = torch.softmax(logits.masked_fill(~visible, float("-inf")), dim=-1)
+        ref[h // (hq // hkv)] += probs[:, :L - N].sum(0)
+    ctx = _ctx(dq, w)
+    scores = torch.empty((hkv, L - N), dtype=torch.float32, device="cuda")
+    dq.dapq_score(ctx, q_win.cuda(), k.cuda(), w.cu_rows, w.prompt_lens, scores)
+    idx = torch.empty((hkv, keep - N), dtype=torch.int32, device="cuda")
+    dq.dapq_topk_select(ctx, scores, w.cu_prompt, w.keep, idx)
+    dq.dapq_poll_status(ctx)
+    util.assert_scores_close(scores.cpu().double().numpy(), ref.numpy(), "prompt window")
+    for h in range(hkv):
+        ref_idx = np.sort(np.argsort(-ref[h].numpy(), kind="stable")[:keep - N])
+        util.assert_index_sets_match(idx[h].cpu().numpy(), ref[h].numpy(), ref_idx, L - N, f"window kvh={h}")
+        kept = np.concatenate([idx[h].cpu().numpy(), np.arange(L - N, L)])      # the caller appends the window rows
+        assert len(np.unique(kept)) == keep
+    dq.dapq_destroy(ctx)
