@@ -207,8 +207,8 @@ dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& 
 dapq_status run_score(dapq_ctx* ctx, int q_dtype, const void* q_rot, const CacheDev& cd, const SeqTable& t,
                       const float* lse_in, float* scores, int64_t score_stride, float* lse_out,
                       float* syn_mass, cudaStream_t s) {
-  cudaError_t e = launch_score_fma(ctx->shape.dtype, q_dtype, q_rot, cd, t, ctx->dims, lse_in, ctx->part, ctx->lse2,
-                                   scores, score_stride, lse_out, syn_mass, s, &ctx->log);
+  cudaError_t e = launch_score_fma(ctx->shape.dtype, q_dtype, q_rot, cd, t, ctx->dims, lse_in, ctx->part, ctx->max_chunks, ctx->n_sm,
+                                   ctx->lse2, scores, score_stride, lse_out, syn_mass, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score kernels");
   return DAPQ_OK;
 }
@@ -270,7 +270,6 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   ctx->dims.n_pseudo = sh->n_pseudo;
   const double scale = sh->softmax_scale > 0.f ? (double)sh->softmax_scale : 1.0 / sqrt((double)kHeadDim);
   ctx->dims.scale_log2e = (float)(scale * 1.4426950408889634074);
-  ctx->max_chunks = (sh->max_total_rows + kChunkKeys - 1) / kChunkKeys + 2LL * sh->max_batch;
 
   DeviceGuard guard(device);
   if (!guard.ok) return bail(DAPQ_ERR_CUDA, "cannot make the device current");
@@ -279,6 +278,10 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
     freq[c] = sh->inv_freq_host ? sh->inv_freq_host[c] : pow(sh->rope_base, -2.0 * c / (double)kHeadDim);
   if (cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || ctx->n_sm < 1)
     return bail(DAPQ_ERR_CUDA, "cannot query the device");
+  // partials of the CUDA-core sweeps: the chunks at 512 keys each, plus room to cut small inputs
+  // finer (down to 64 keys) until every SM has two CTAs
+  ctx->max_chunks = (sh->max_total_rows + kChunkKeys - 1) / kChunkKeys + 2LL * sh->max_batch +
+                    (2LL * ctx->n_sm + sh->n_kv_heads - 1) / sh->n_kv_heads;
   const size_t hq_n = (size_t)sh->n_q_heads * sh->n_pseudo;
   ctx->q_rows_max = (int64_t)sh->max_batch * hq_n;
   size_t part_elems = (size_t)ctx->max_chunks * hq_n;

@@ -12,7 +12,7 @@ namespace dapq {
 constexpr int kHeadDim = DAPQ_HEAD_DIM;      // d
 constexpr int kMaxBatch = DAPQ_MAX_BATCH;
 constexpr int kMaxPseudo = DAPQ_MAX_PSEUDO;
-constexpr int kChunkKeys = 512;              // prompt keys per work chunk of the score sweeps
+constexpr int kChunkKeys = 512;              // most prompt keys per work chunk of the CUDA-core score sweeps
 
 // Per-call sequence geometry, passed by value to the kernels (host arrays never have to
 // be copied to the device, so a call adds no copy nodes to a stream).
@@ -26,7 +26,8 @@ struct SeqTable {
 };
 
 // How the score sweeps cut the sequences into work chunks (one CTA per chunk and KV head).
-//   CUDA-core path:   chunks of kChunkKeys prompt keys, then one chunk with the N synthetic rows;
+//   CUDA-core path:   chunks of chunk_tiles prompt KEYS (64 .. kChunkKeys), then one chunk with the N
+//                     synthetic rows;
 //   tensor-core path: chunks of chunk_tiles whole K tiles (the tile size is the sweep's).
 struct ChunkTable {
   int32_t chunk_tiles;
@@ -121,11 +122,13 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
                         const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log);
 
 // Generic CUDA-core scorer (any N <= 128, both dtypes).
-//   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits
+//   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits, room for max_chunks
+//           chunks (at least the count at kChunkKeys keys per chunk; more lets small inputs
+//           be cut finer so that they fill the n_sm SMs)
 //   lse2  : [B, H_q, N] base-2 log-sum-exp
 cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
-                             const Dims& dm, const float* lse_in, float2* part, float* lse2,
-                             float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
+                             const Dims& dm, const float* lse_in, float2* part, int64_t max_chunks, int n_sm,
+                             float* lse2, float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
                              cudaStream_t s, LaunchLog* log);
 
 // Tensor-core scorer (bf16 caches).  umma_plan encodes the TMA descriptors and cuts the work;

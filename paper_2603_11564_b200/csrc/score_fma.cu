@@ -71,8 +71,10 @@ constexpr size_t fma_smem_bytes() {
   return sizeof(float) * (size_t)(16 * R * kPad + kTileKeys * kPad + 8 * kTileKeys + kChunkKeys + 16 * R);
 }
 
-// grid (n_chunks, H_kv).  Thread (ty, tx) owns query rows ty + 16 r (r < R) and the keys
-// kk * 16 + tx (kk < 4) of each 64-key tile.
+// grid (n_chunks, H_kv) in sweep 2, which sums over the G heads of the group in a fixed order;
+// (n_chunks, H_kv, G) in sweep 1, whose partials are per head.  A chunk holds ct.chunk_tiles
+// prompt keys (64 .. kChunkKeys, chosen per call).  Thread (ty, tx) owns query rows ty + 16 r
+// (r < R) and the keys kk * 16 + tx (kk < 4) of each 64-key tile.
 template <typename TQ, typename T, int R, bool kSweep2>
 __global__ void __launch_bounds__(kThreads)
 score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_constant__ SeqTable t,
@@ -87,11 +89,11 @@ score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_c
 
   const int chunk = blockIdx.x, kvh = blockIdx.y, tid = threadIdx.x;
   const int b = find_segment(ct.cu_chunk, t.batch, chunk);
-  const int c = chunk - ct.cu_chunk[b];
+  const int c = chunk - ct.cu_chunk[b], chunk_keys = ct.chunk_tiles;
   const int L = t.prompt_len[b], N = dm.n_pseudo, G = dm.group, Hq = dm.n_q_heads;
   const bool syn = (c == ct.cu_chunk[b + 1] - ct.cu_chunk[b] - 1);
-  const int key_begin = syn ? L : c * kChunkKeys;
-  const int key_end = syn ? L + N : min(L, key_begin + kChunkKeys);
+  const int key_begin = syn ? L : c * chunk_keys;
+  const int key_end = syn ? L + N : min(L, key_begin + chunk_keys);
   if (kSweep2 && syn && syn_mass == nullptr) return;
 
   const T* kbase = reinterpret_cast<const T*>(cv.k) + (int64_t)kvh * cv.k_head_stride +
@@ -102,7 +104,8 @@ score_fma_kernel(const TQ* __restrict__ q_rot, const CacheDev cv, const __grid_c
     for (int x = tid; x < kChunkKeys; x += kThreads) colacc[x] = 0.f;
   }
 
-  for (int g = 0; g < G; ++g) {
+  const int g_begin = kSweep2 ? 0 : (int)blockIdx.z, g_end = kSweep2 ? G : g_begin + 1;
+  for (int g = g_begin; g < g_end; ++g) {
     const int h = kvh * G + g;
     __syncthreads();                                        // Qs, lse_s, colacc free
     stage_rows<TQ>(Qs, q_rot + ((int64_t)b * Hq + h) * N * kHeadDim, kHeadDim, N, 16 * R);
@@ -258,7 +261,7 @@ __global__ void lse_import_kernel(const float* __restrict__ lse_in, int n, float
 
 template <typename TQ, typename T, int R>
 cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, const Dims& dm,
-                    const float* lse_in, float2* part, float* lse2, float* scores,
+                    const float* lse_in, float2* part, int64_t max_chunks, int n_sm, float* lse2, float* scores,
                     int64_t score_stride, float* lse_out, float* syn_mass, cudaStream_t s,
                     LaunchLog* log) {
   constexpr size_t smem = fma_smem_bytes<R>();
@@ -267,20 +270,29 @@ cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, co
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  // Keys per chunk: the largest of 512 .. 64 that gives every SM two CTAs in sweep 2, else the
+  // smallest whose partials fit the caller's buffer (512 always fits: the callers check it).
   ChunkTable ct;
-  ct.chunk_tiles = 0;
+  ct.chunk_tiles = kChunkKeys;
   int32_t n_chunks = 0;
-  for (int b = 0; b < t.batch; ++b) {
-    ct.cu_chunk[b] = n_chunks;
-    n_chunks += (t.prompt_len[b] + kChunkKeys - 1) / kChunkKeys + 1;
+  for (int ck = kChunkKeys; ck >= kTileKeys; ck >>= 1) {
+    int64_t n = 0;
+    for (int b = 0; b < t.batch; ++b) n += (t.prompt_len[b] + ck - 1) / ck + 1;
+    if (ck < kChunkKeys && n > max_chunks) break;
+    ct.chunk_tiles = ck;
+    n_chunks = (int32_t)n;
+    if (n * dm.n_kv_heads >= 2LL * n_sm) break;
   }
-  ct.cu_chunk[t.batch] = n_chunks;
+  for (int b = 0, n = 0; b <= t.batch; ++b) {
+    ct.cu_chunk[b] = n;
+    if (b < t.batch) n += (t.prompt_len[b] + ct.chunk_tiles - 1) / ct.chunk_tiles + 1;
+  }
   ct.n_chunks = n_chunks;
-  const dim3 grid(n_chunks, dm.n_kv_heads);
+  const dim3 grid(n_chunks, dm.n_kv_heads), grid1(n_chunks, dm.n_kv_heads, dm.group);
   const int n_lse = t.batch * dm.n_q_heads * dm.n_pseudo;
   if (lse_in == nullptr) {
     log->begin(kKindSweep1, s);
-    k1<<<grid, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, ct, dm, part, nullptr, nullptr, 0, nullptr);
+    k1<<<grid1, kThreads, smem, s>>>((const TQ*)q_rot, cv, t, ct, dm, part, nullptr, nullptr, 0, nullptr);
     log->end(s);
     log->begin(kKindLseMerge, s);
     lse_merge_kernel<<<(n_lse + 127) / 128, 128, 0, s>>>(part, t, ct, dm.n_q_heads, dm.n_pseudo, lse2, lse_out);
@@ -298,27 +310,27 @@ cudaError_t run_fma(const void* q_rot, const CacheDev& cv, const SeqTable& t, co
 
 template <typename TQ, typename T>
 cudaError_t run_fma_n(const void* q_rot, const CacheDev& cv, const SeqTable& t, const Dims& dm,
-                      const float* lse_in, float2* part, float* lse2, float* scores,
+                      const float* lse_in, float2* part, int64_t max_chunks, int n_sm, float* lse2, float* scores,
                       int64_t score_stride, float* lse_out, float* syn_mass, cudaStream_t s,
                       LaunchLog* log) {
   const int n = dm.n_pseudo;
-  if (n <= 16) return run_fma<TQ, T, 1>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
-  if (n <= 32) return run_fma<TQ, T, 2>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
-  if (n <= 64) return run_fma<TQ, T, 4>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
-  return run_fma<TQ, T, 8>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  if (n <= 16) return run_fma<TQ, T, 1>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  if (n <= 32) return run_fma<TQ, T, 2>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  if (n <= 64) return run_fma<TQ, T, 4>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  return run_fma<TQ, T, 8>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
 }
 
 }  // namespace
 
 cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
-                             const Dims& dm, const float* lse_in, float2* part, float* lse2,
-                             float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
+                             const Dims& dm, const float* lse_in, float2* part, int64_t max_chunks, int n_sm,
+                             float* lse2, float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
                              cudaStream_t s, LaunchLog* log) {
   if (dtype == DAPQ_BF16 && q_dtype == DAPQ_BF16)
-    return run_fma_n<__nv_bfloat16, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+    return run_fma_n<__nv_bfloat16, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
   if (dtype == DAPQ_BF16)
-    return run_fma_n<float, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
-  return run_fma_n<float, float>(q_rot, cv, t, dm, lse_in, part, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+    return run_fma_n<float, __nv_bfloat16>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
+  return run_fma_n<float, float>(q_rot, cv, t, dm, lse_in, part, max_chunks, n_sm, lse2, scores, score_stride, lse_out, syn_mass, s, log);
 }
 
 }  // namespace dapq

@@ -96,15 +96,17 @@ extern "C" dapq_status dapq_score_static(const dapq_shape* sh, int device, const
   }
   t.cu_prompt[cv->batch] = (int32_t)prompt;
   t.cu_keep[cv->batch] = (int32_t)prompt;
+  // layout of the fixed area: the base-2 lse [B, H_q, N] first, the sweeps' partials after it
   const size_t hq_n = (size_t)sh->n_q_heads * sh->n_pseudo;
-  const size_t part_bytes = (size_t)chunks * hq_n * sizeof(float2);
-  const size_t lse_off = (part_bytes + 255) & ~(size_t)255;
-  const size_t need = lse_off + (size_t)cv->batch * hq_n * sizeof(float);
+  const size_t part_off = ((size_t)cv->batch * hq_n * sizeof(float) + 255) & ~(size_t)255;
+  const size_t need = part_off + (size_t)chunks * hq_n * sizeof(float2);
   if (need > (size_t)DAPQ_STATIC_SCRATCH_BYTES)
     return fail_static(err, err_len, DAPQ_ERR_WORKSPACE,
                        "dapq_score_static: this call needs %zu bytes of scratch, the fixed area holds %d "
                        "(chunks of 512 keys x H_q x N x 8 bytes); use dapq_create + dapq_score for larger caches",
                        need, (int)DAPQ_STATIC_SCRATCH_BYTES);
+  // what is left lets the launcher cut small inputs into finer chunks
+  const int64_t max_chunks = (int64_t)(((size_t)DAPQ_STATIC_SCRATCH_BYTES - part_off) / (hq_n * sizeof(float2)));
 
   DeviceScope scope(device);
   if (!scope.ok) return fail_static(err, err_len, DAPQ_ERR_CUDA, "cannot make device %d current", device);
@@ -137,10 +139,13 @@ extern "C" dapq_status dapq_score_static(const dapq_shape* sh, int device, const
   cd.v_head_stride = cd.v_row_stride = 0;
   // Every partial and every lse entry the second sweep reads is written by this call first,
   // so nothing left in the area by an earlier call has to be cleared.
-  float2* part = reinterpret_cast<float2*>(base);
-  float* lse2 = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + lse_off);
+  float* lse2 = reinterpret_cast<float*>(base);
+  float2* part = reinterpret_cast<float2*>(static_cast<unsigned char*>(base) + part_off);
+  int n_sm = 0;
+  if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n_sm < 1)
+    return fail_static(err, err_len, DAPQ_ERR_CUDA, "cannot query device %d", device);
   LaunchLog log;
-  const cudaError_t e = launch_score_fma(sh->dtype, sh->dtype, q_rot, cd, t, dm, nullptr, part, lse2, scores,
+  const cudaError_t e = launch_score_fma(sh->dtype, sh->dtype, q_rot, cd, t, dm, nullptr, part, max_chunks, n_sm, lse2, scores,
                                          (int64_t)prompt, nullptr, nullptr, (cudaStream_t)stream, &log);
   if (e != cudaSuccess) return fail_static(err, err_len, DAPQ_ERR_CUDA, "score kernels: %s", cudaGetErrorString(e));
   return DAPQ_OK;

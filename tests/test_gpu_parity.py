@@ -97,6 +97,10 @@ SCORE_CASES = [
     ("bf16", 8, 1, 128, (129, 1031)),
     ("bf16", 4, 4, 100, (777,)),
     ("bf16", 8, 2, 17, (512, 1024, 300, 5)),
+    # CUDA-core sweeps at every chunk size (512 / 256 / 128 keys on a 148-SM part; the shorter cases above take 64)
+    ("f32", 8, 8, 8, (19000,)),
+    ("bf16", 8, 8, 4, (9000, 700)),
+    ("f32", 4, 4, 16, (9500,)),
 ]
 
 
