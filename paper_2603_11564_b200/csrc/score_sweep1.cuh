@@ -4,7 +4,8 @@
 //
 //   D[query, key] = Q_blk K_tile^T, queries on tensor-memory lanes, 192 keys per tile.
 // A job is one [128 queries x 192 keys] accumulator; the two query blocks of a group own one
-// accumulator each, so the MMAs of one block run while the other block's accumulator is read.
+// accumulator each, so the MMAs of one block run while the other block's accumulator is read
+// (a group of one block alternates between the two accumulators from tile to tile).
 // All four epilogue groups work on every job, 48 key columns each: thread (group g, row r) keeps
 // the statistics of query row r over the columns of its group, which become slot g of the
 // row's per-chunk partials.  Sixteen epilogue warps (four per scheduler) hide the latency of
@@ -63,6 +64,7 @@ __device__ __forceinline__ void row_stats_job(uint32_t taddr, int col0, bool mas
   }
 }
 
+template <bool kCompact>
 __global__ void __launch_bounds__(kThreads, 1)
 score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                     const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct, const UmmaArgs a) {
@@ -70,17 +72,19 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  using G = Geo<kCompact>;
+  constexpr int kStages1 = G::kStages1;
   const int chunk = blockIdx.x, kvh = blockIdx.y;
   const Work w = cta_work(t, ct, a, kTile1, true);
   const int nt = w.nt, L = w.L, N = a.n_pseudo;
   if (nt <= 0) return;
   const Bars bars{sbase + Smem::bars};
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
-  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages1);
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages1, 2);
 
   if (warp == 0) {
     if (lane == 0)
-      tma_producer<kTile1, kStages1, kStageBytes1, kHalfBytes1>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
+      tma_producer<G, kTile1, kStages1, kStageBytes1, kHalfBytes1>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
@@ -88,16 +92,16 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       uint32_t use0 = 0u, use1 = 0u;                            // jobs issued into each accumulator
       bool ok = true;
       const uint32_t idesc = umma_idesc(128, kTile1);
-      const uint64_t qd_hi = umma_desc(sbase + Smem::q_hi), qd_lo = umma_desc(sbase + Smem::q_lo);
+      const uint64_t qd_hi = umma_desc(sbase + G::q_hi), qd_lo = umma_desc(sbase + G::q_lo);
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
-        const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+        const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
         const int mb = (rows_g + 127) / 128;
         ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
         for (int ti = 0; ti < nt && ok; ++ti, ++li) {
           const int s = li % kStages1;
           ok = mbar_wait(bars.k_full(s), (li / kStages1) & 1, abort_flag, a.status);
           if (!ok) break;
-          const uint64_t kd = umma_desc(sbase + Smem::k + s * kStageBytes1);
+          const uint64_t kd = umma_desc(sbase + G::k + s * kStageBytes1);
           for (int m = 0; m < mb && ok; ++m) {
             // two blocks: block m -> accumulator m; one block: tiles alternate between the two
             const int buf = (mb == 2) ? m : (ti & 1);
@@ -110,14 +114,14 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const int half = ks >> 2, kk = ks & 3;
-              umma_ss(d, desc_advance(qh, half * kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
+              umma_ss(d, desc_advance(qh, half * G::kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
                       idesc, ks ? 1u : 0u);
             }
             if (a.has_lo) {
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
                 const int half = ks >> 2, kk = ks & 3;
-                umma_ss(d, desc_advance(ql, half * kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
+                umma_ss(d, desc_advance(ql, half * G::kHalfBytesQ + kk * 32), desc_advance(kd, half * kHalfBytes1 + kk * 32),
                         idesc, 1u);
               }
             }
@@ -140,11 +144,11 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     uint32_t use0 = 0u, use1 = 0u;                              // jobs taken from each accumulator
     bool ok = true;
     for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
-      const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+      const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
       const int mb = (rows_g + 127) / 128;
       // running max (raw dot product) and sum of this thread's row of block 0 / block 1
       float m_raw0 = -CUDART_INF_F, z0 = 0.f, m_raw1 = -CUDART_INF_F, z1 = 0.f;
-      const int i_q0 = (qg * kGroupRows + r) % N, i_q1 = (qg * kGroupRows + 128 + r) % N;   // pseudo-query indices
+      const int i_q0 = (qg * G::kRows + r) % N, i_q1 = (qg * G::kRows + 128 + r) % N;   // pseudo-query indices
       for (int ti = 0; ti < nt && ok; ++ti) {
         const int tile_base = (w.t0 + ti) * kTile1;
         const bool masked = tile_base + kTile1 > L;             // holds synthetic (or foreign) rows
@@ -165,10 +169,9 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
       }
       // partials: slot eg of this thread's rows
-      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * kEpiGroups + eg) * (a.n_qgroups * kGroupRows) +
-                      qg * kGroupRows;
-      if (qg * kGroupRows + r < a.rows_total) pbase[r] = make_float2(m_raw0 * c, z0);
-      if (mb == 2 && qg * kGroupRows + 128 + r < a.rows_total) pbase[128 + r] = make_float2(m_raw1 * c, z1);
+      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * kEpiGroups + eg) * a.rows_pad + qg * G::kRows;
+      if (qg * G::kRows + r < a.rows_total) pbase[r] = make_float2(m_raw0 * c, z0);
+      if (mb == 2 && qg * G::kRows + 128 + r < a.rows_total) pbase[128 + r] = make_float2(m_raw1 * c, z1);
     }
   }
   cta_epilogue(tmem_base);

@@ -2,10 +2,12 @@
 // summed over the N pseudo queries and the G query heads of the KV head's group.
 //
 //   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
-// A job is one [128 keys x 256 queries] accumulator (two fit).  All four epilogue groups work
+// A job is one [128 keys x 256 queries] accumulator (two fit; four of 128 columns in the compact
+// geometry).  All four epilogue groups work
 // on every job, a quarter of the query columns each (sixteen epilogue warps, four per scheduler,
-// hide the latency of the tensor-memory loads and of the hand-offs); groups 1-3 hand their
-// partial sums to group 0 through consumed columns of the same accumulator, and group 0's thread
+// hide the latency of the tensor-memory loads and of the hand-offs); three groups hand their
+// partial sums to the fourth through consumed columns of the same accumulator (the groups take
+// that part in turn, job by job, so none of them lags behind), and that group's thread
 // (lane = key) stores the key's score: one coalesced fp32 per lane.  Before the first job the
 // epilogue threads merge the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the
 // resident query rows.
@@ -15,6 +17,7 @@
 namespace dapq {
 namespace umma {
 
+template <bool kCompact>
 __global__ void __launch_bounds__(kThreads, 1)
 score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                     const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
@@ -23,6 +26,8 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  using G = Geo<kCompact>;
+  constexpr int kStages2 = G::kStages2, kAcc = G::kAcc2, kAccCols = G::kAccCols2;
   const int chunk = blockIdx.x, kvh = blockIdx.y;
   const Work w = cta_work(t, ct, a, kTile2, false);
   const int nt = w.nt, L = w.L, b = w.b;
@@ -30,40 +35,40 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   const Bars bars{sbase + Smem::bars};
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
   float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
-  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages2);
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages2, kAcc);
 
   if (warp == 0) {
     if (lane == 0)
-      tma_producer<kTile2, kStages2, kStageBytes2, kHalfBytes2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
+      tma_producer<G, kTile2, kStages2, kStageBytes2, kHalfBytes2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
       int job = 0;                                              // = K tiles consumed: one job per tile
       bool ok = true;
-      const uint64_t qd_hi = umma_desc(sbase + Smem::q_hi), qd_lo = umma_desc(sbase + Smem::q_lo);
+      const uint64_t qd_hi = umma_desc(sbase + G::q_hi), qd_lo = umma_desc(sbase + G::q_lo);
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
-        const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+        const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
         const uint32_t idesc = umma_idesc(128, (rows_g + 15) & ~15);   // only the query columns that exist
         ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
         for (int ti = 0; ti < nt && ok; ++ti, ++job) {
-          const int s = job % kStages2, buf = job & 1;
+          const int s = job % kStages2, buf = job % kAcc;
           ok = mbar_wait(bars.k_full(s), (job / kStages2) & 1, abort_flag, a.status);
-          if (ok && job >= 2) ok = mbar_wait(bars.acc_empty(buf), ((job >> 1) - 1) & 1, abort_flag, a.status);
+          if (ok && job >= kAcc) ok = mbar_wait(bars.acc_empty(buf), ((job / kAcc) - 1) & 1, abort_flag, a.status);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t kd = umma_desc(sbase + Smem::k + s * kStageBytes2);
-          const uint32_t d = tmem_base + buf * 256;
+          const uint64_t kd = umma_desc(sbase + G::k + s * kStageBytes2);
+          const uint32_t d = tmem_base + buf * kAccCols;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const int half = ks >> 2, kk = ks & 3;
-            umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * kHalfBytesQ + kk * 32),
+            umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * G::kHalfBytesQ + kk * 32),
                     idesc, ks ? 1u : 0u);
           }
           if (a.has_lo) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const int half = ks >> 2, kk = ks & 3;
-              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_lo, half * kHalfBytesQ + kk * 32),
+              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_lo, half * G::kHalfBytesQ + kk * 32),
                       idesc, 1u);
             }
           }
@@ -85,18 +90,18 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     bool ok = true;
     // (an aborting group still walks every query group: the other groups wait for it at the barriers)
     for (int qg = 0; qg < a.n_qgroups; ++qg) {
-      const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+      const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
       // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk
       // partials of row eg*128 + r in a fixed order, or converts the caller's value
       if (qg > 0) epilogue_sync();                              // the previous group's values are no longer read
-      if (eg < 2) {
-        const int row = eg * 128 + r, grow = qg * kGroupRows + row;
+      if (eg * 128 < G::kRows) {
+        const int row = eg * 128 + r, grow = qg * G::kRows + row;
         float l2 = 0.f;
         if (grow < a.rows_total) {
           if (a.lse_in) {
             l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
           } else {
-            const int rows_pad = a.n_qgroups * kGroupRows;
+            const int rows_pad = a.rows_pad;
             const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * kEpiGroups * rows_pad + grow;
             const int64_t step = (int64_t)a.n_kv_heads * kEpiGroups * rows_pad;
             const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
@@ -132,11 +137,11 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       const int nch = (rows_g + 31) >> 5;
       const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
       for (int ti = 0; ti < nt && ok; ++ti, ++job) {
-        const int buf = job & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), (job >> 1) & 1, abort_flag, a.status));
+        const int buf = job % kAcc;
+        ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), (job / kAcc) & 1, abort_flag, a.status));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = lane_addr + buf * 256;
+        const uint32_t taddr = lane_addr + buf * kAccCols;
         float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
@@ -166,7 +171,8 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           }
         }
         float sum = (acc.x + acc.y) + (acc1.x + acc1.y);
-        if (eg > 0) {
+        const int red = job % kEpiGroups;                       // the group that sums this job's partials: each in turn
+        if (eg != red) {
           // hand the partial sum over in the first column this group has consumed (nothing to hand over
           // if it had no columns), then release the accumulator
           if (np > 0) {
@@ -177,18 +183,19 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           __syncwarp();
           if (lane == 0) { mbar_arrive(bars.half_done(buf)); mbar_arrive(bars.acc_empty(buf)); }
         } else {
-          ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job >> 1) & 1, abort_flag, a.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job / kAcc) & 1, abort_flag, a.status));
           if (!ok) break;
           tc_fence_after();
-          // the three partial sums: loads issued together, one wait (a group without columns left nothing)
-          uint32_t part[kEpiGroups - 1] = {0u, 0u, 0u};
+          // the other groups' partial sums: loads issued together, one wait (a group without columns left
+          // nothing); own slot and empty slots stay zero, the order of the additions is fixed
+          uint32_t part[kEpiGroups] = {0u, 0u, 0u, 0u};
 #pragma unroll
-          for (int g = 1; g < kEpiGroups; ++g) {
+          for (int g = 0; g < kEpiGroups; ++g) {
             const int gp0 = (g * nch) / kEpiGroups, gnp = ((g + 1) * nch) / kEpiGroups - gp0;
-            if (gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g - 1]);
+            if (g != eg && gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g]);
           }
-          tmem_ld_wait3(part[0], part[1], part[2]);
-          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + __uint_as_float(part[2]);
+          tmem_ld_wait4(part[0], part[1], part[2], part[3]);
+          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + (__uint_as_float(part[2]) + __uint_as_float(part[3]));
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.acc_empty(buf));

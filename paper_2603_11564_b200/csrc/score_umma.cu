@@ -13,6 +13,9 @@
 //             running max / sum of exp of every pseudo query;
 //   sweep 2 (score_sweep2.cuh)  keys on lanes, up to 256 query columns per MMA: merges the
 //             partials into each query's log-sum-exp, then sums exp2(s - lse_i) per key.
+// When the G*N rows of a KV head fit one block of 128 (N = 32 with G = 4) both sweeps run in a
+// compact geometry: half the shared memory for the queries, a deeper K ring, and four
+// accumulators of 128 columns in sweep 2.
 // The rotated queries are used as a bf16 pair (hi + lo, lo = bf16(q - hi)): two MMAs per
 // k-step with the same K tile.  A single bf16 rounding of q would put the per-token scores
 // of caches with outlier channels outside the 2e-3 tolerance.
@@ -106,7 +109,7 @@ bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int n_kv_head
 
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo) {
   const int rows_total = n_q_heads / n_kv_heads * n_pseudo;
-  const int rows_pad = (rows_total + kGroupRows - 1) / kGroupRows * kGroupRows;
+  const int rows_pad = (rows_total + 255) / 256 * 256;          // (the compact geometry pads to 128: never more)
   return (int64_t)(max_batch + kUmmaMaxChunks) * n_kv_heads * kEpiGroups * rows_pad;
 }
 
@@ -138,7 +141,10 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   a.n_q_heads = dm.n_q_heads;
   a.n_kv_heads = dm.n_kv_heads;
   a.rows_total = dm.group * dm.n_pseudo;
-  a.n_qgroups = (a.rows_total + kGroupRows - 1) / kGroupRows;
+  const bool compact = a.rows_total <= Geo<true>::kRows;
+  const int group_rows = compact ? Geo<true>::kRows : Geo<false>::kRows;
+  a.n_qgroups = (a.rows_total + group_rows - 1) / group_rows;
+  a.rows_pad = a.n_qgroups * group_rows;
   a.has_lo = plan.has_lo;
   a.lo_row_offset = (int32_t)plan.lo_row_offset;
   a.scale_log2e = dm.scale_log2e;
@@ -149,19 +155,25 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   a.score_stride = score_stride;
   a.status = status;
 
-  cudaError_t e;
-  if ((e = cudaFuncSetAttribute(score_sweep1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(score_sweep2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
-  if (lse_in == nullptr) {
-    log->begin(kKindSweep1, s);
-    launch_pdl(score_sweep1_kernel, dim3(plan.ct1.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k1,
-               plan.tm_q, t, plan.ct1, a);
+  auto run = [&](auto sweep1, auto sweep2) -> cudaError_t {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(sweep1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(sweep2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
+    if (lse_in == nullptr) {
+      log->begin(kKindSweep1, s);
+      launch_pdl(sweep1, dim3(plan.ct1.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k1, plan.tm_q, t,
+                 plan.ct1, a);
+      log->end(s);
+    }
+    log->begin(kKindSweep2, s);
+    launch_pdl(sweep2, dim3(plan.ct2.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k2, plan.tm_q, t,
+               plan.ct2, plan.ct1, a);
     log->end(s);
-  }
-  log->begin(kKindSweep2, s);
-  launch_pdl(score_sweep2_kernel, dim3(plan.ct2.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k2,
-             plan.tm_q, t, plan.ct2, plan.ct1, a);
-  log->end(s);
+    return cudaSuccess;
+  };
+  const cudaError_t e = compact ? run(score_sweep1_kernel<true>, score_sweep2_kernel<true>)
+                                : run(score_sweep1_kernel<false>, score_sweep2_kernel<false>);
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 

@@ -9,41 +9,58 @@ using namespace ptx;
 
 constexpr int kTile1 = 192;                    // keys per K tile of sweep 1 (= UMMA N there)
 constexpr int kTile2 = 128;                    // keys per K tile of sweep 2 (= UMMA M there)
-constexpr int kGroupRows = 256;                // query rows resident per group (2 blocks of 128)
-constexpr int kHalfBytesQ = kGroupRows * 128;  // one 64-channel half of a query group (32 KB)
-constexpr int kQBytes = 2 * kHalfBytesQ;       // 64 KB per precision part (hi / lo)
 constexpr int kEpiGroups = 4;                  // epilogue groups of 4 warps (128 TMEM lanes each)
 constexpr int kThreads = 64 + kEpiGroups * 128;
 constexpr int kTmemCols = 512;
+constexpr int kStageBytes1 = kTile1 * 256, kHalfBytes1 = kTile1 * 128;   // one K tile of sweep 1 / its 64-channel half
+constexpr int kStageBytes2 = kTile2 * 256, kHalfBytes2 = kTile2 * 128;
 
-// Shared memory of both sweeps (offsets from the 1024-aligned base): the query group as a
-// bf16 pair, a K ring of 96 KB (2 x 192 keys in sweep 1, 3 x 128 keys in sweep 2), barriers,
-// and (sweep 2) the group's log-sum-exp.
-constexpr int kStages1 = 2, kStageBytes1 = kTile1 * 256, kHalfBytes1 = kTile1 * 128;
-constexpr int kStages2 = 3, kStageBytes2 = kTile2 * 256, kHalfBytes2 = kTile2 * 128;
-struct Smem {
+// Geometry of a CTA.  kCompact = the G*N query rows of a KV head fit one block of 128 (the
+// paper's default window, N = 32 with four query heads per KV head): the query operand then
+// takes 64 KB instead of 128 KB, the K ring grows from 96 KB to 160 KB, and sweep 2 runs four
+// accumulators of 128 columns instead of two of 256.
+template <bool kCompact>
+struct Geo {
+  static constexpr int kRows = kCompact ? 128 : 256;          // query rows resident per group
+  static constexpr int kHalfBytesQ = kRows * 128;             // one 64-channel half of a query group
+  static constexpr int kQBytes = 2 * kHalfBytesQ;             // per precision part (hi / lo)
+  static constexpr int kRingBytes = 224 * 1024 - 2 * kQBytes;
+  static constexpr int kStages1 = kRingBytes / kStageBytes1;  // 2 / 3 tiles of 192 keys
+  static constexpr int kStages2 = kRingBytes / kStageBytes2;  // 3 / 5 tiles of 128 keys
+  static constexpr int kAcc2 = kCompact ? 4 : 2;              // accumulators of sweep 2
+  static constexpr int kAccCols2 = kTmemCols / kAcc2;
+  // shared memory (offsets from the 1024-aligned base): query group as a bf16 pair, K ring
   static constexpr int q_hi = 0;
-  static constexpr int q_lo = q_hi + kQBytes;
-  static constexpr int k = q_lo + kQBytes;
-  static constexpr int bars = k + 96 * 1024;
-  // barriers (16 x 8 B): k_full[3], k_empty[3], acc_full[2], acc_empty[2], q_full, q_empty, half_done[2]
-  static constexpr int lse = bars + 16 * 8;          // [256] floats
-  static constexpr int tmem_ptr = lse + kGroupRows * 4;
+  static constexpr int q_lo = kQBytes;
+  static constexpr int k = 2 * kQBytes;
+};
+constexpr int kMaxStages = 5, kMaxAcc = 4;
+// ... followed, at the same place in both geometries, by the barriers, the group's log-sum-exp
+// (sweep 2) and two words.
+struct Smem {
+  static constexpr int bars = 224 * 1024;
+  // barriers (24 x 8 B): k_full[5], k_empty[5], acc_full[4], acc_empty[4], q_full, q_empty, half_done[4]
+  static constexpr int lse = bars + 24 * 8;          // [256] floats
+  static constexpr int tmem_ptr = lse + 256 * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
-static_assert(kStages1 * kStageBytes1 == 96 * 1024 && kStages2 * kStageBytes2 == 96 * 1024, "K ring is 96 KB");
+static_assert(Geo<false>::k + Geo<false>::kStages1 * kStageBytes1 <= Smem::bars && Geo<true>::k + Geo<true>::kStages1 * kStageBytes1 <= Smem::bars &&
+              Geo<false>::k + Geo<false>::kStages2 * kStageBytes2 <= Smem::bars && Geo<true>::k + Geo<true>::kStages2 * kStageBytes2 <= Smem::bars,
+              "K ring overruns the barriers");
+static_assert(Geo<true>::kStages2 <= kMaxStages && Geo<true>::kAcc2 <= kMaxAcc, "barrier table too small");
 constexpr int kSmemBytes = Smem::total + 1024;   // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
 struct UmmaArgs {
   int32_t n_pseudo, group, n_q_heads, n_kv_heads;
   int32_t rows_total;        // G * N
-  int32_t n_qgroups;         // ceil(rows_total / 256)
+  int32_t n_qgroups;         // ceil(rows_total / rows per group)
+  int32_t rows_pad;          // n_qgroups * rows per group
   int32_t has_lo;            // the query operand carries a low-order bf16 part
   int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
   float scale_log2e;
-  float2* part;              // [n_chunks1, H_kv, 4, n_qgroups * 256] (running max, sum) in base 2, one slot per group
+  float2* part;              // [n_chunks1, H_kv, 4, rows_pad] (running max, sum) in base 2, one slot per group
   const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
   float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
   float* scores;
@@ -75,25 +92,25 @@ __device__ __forceinline__ Work cta_work(const SeqTable& t, const ChunkTable& ct
 struct Bars {
   uint32_t base;
   __device__ __forceinline__ uint32_t k_full(int s) const { return base + 8u * s; }
-  __device__ __forceinline__ uint32_t k_empty(int s) const { return base + 8u * (3 + s); }
-  __device__ __forceinline__ uint32_t acc_full(int i) const { return base + 8u * (6 + i); }
-  __device__ __forceinline__ uint32_t acc_empty(int i) const { return base + 8u * (8 + i); }
-  __device__ __forceinline__ uint32_t q_full() const { return base + 8u * 10; }
-  __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * 11; }
-  __device__ __forceinline__ uint32_t half_done(int i) const { return base + 8u * (12 + i); }
+  __device__ __forceinline__ uint32_t k_empty(int s) const { return base + 8u * (kMaxStages + s); }
+  __device__ __forceinline__ uint32_t acc_full(int i) const { return base + 8u * (2 * kMaxStages + i); }
+  __device__ __forceinline__ uint32_t acc_empty(int i) const { return base + 8u * (2 * kMaxStages + kMaxAcc + i); }
+  __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc); }
+  __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 1); }
+  __device__ __forceinline__ uint32_t half_done(int i) const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 2 + i); }
 };
 
 // Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync, then
 // the wait for the kernel before this one (its set-up overlaps that kernel's tail).
 // Returns the tensor-memory base address.
-__device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, int n_stages) {
+__device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, int n_stages, int n_acc) {
   const int warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(bars.k_full(s), 1); mbar_init(bars.k_empty(s), 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < n_acc; ++i) {
       mbar_init(bars.acc_full(i), 1);
       mbar_init(bars.acc_empty(i), 4 * kEpiGroups);        // every epilogue warp reads every accumulator
-      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the groups that hand their partial sums to group 0
+      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the three groups that hand their partial sums over
     }
     mbar_init(bars.q_full(), 1);
     mbar_init(bars.q_empty(), 1);
@@ -123,7 +140,7 @@ __device__ __forceinline__ void cta_epilogue(uint32_t tmem_base) {
 
 // TMA producer loop shared by both sweeps: per query group the query blocks (hi, lo), then the
 // CTA's K tiles through the ring.  kTile / kStages / kHalf are the sweep's tile geometry.
-template <int kTile, int kStages, int kStage, int kHalf>
+template <class G, int kTile, int kStages, int kStage, int kHalf>
 __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w,
                                              const UmmaArgs& a, uint32_t sbase, const Bars& bars, int kvh,
                                              volatile int* abort_flag) {
@@ -133,15 +150,15 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     const int s = li % kStages;
     mbar_expect_tx(bars.k_full(s), kStage);
     const int row = w.row_base + (w.t0 + ti) * kTile;
-    tma_load_3d(sbase + Smem::k + s * kStage, tm_k, bars.k_full(s), 0, row, kvh);
-    tma_load_3d(sbase + Smem::k + s * kStage + kHalf, tm_k, bars.k_full(s), 64, row, kvh);
+    tma_load_3d(sbase + G::k + s * kStage, tm_k, bars.k_full(s), 0, row, kvh);
+    tma_load_3d(sbase + G::k + s * kStage + kHalf, tm_k, bars.k_full(s), 64, row, kvh);
     ++li;
   };
   // The first K tiles go out before the queries: they come from further away (DRAM in sweep 1).
   const int n_first = min(kStages, w.nt);
   for (int ti = 0; ti < n_first; ++ti) load_tile(ti);
   for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
-    const int rows_g = min(kGroupRows, a.rows_total - qg * kGroupRows);
+    const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
     const int mb = (rows_g + 127) / 128;
     if (qg > 0) ok = mbar_wait(bars.q_empty(), (qg - 1) & 1, abort_flag, a.status);
     if (!ok) break;
@@ -150,8 +167,8 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     for (int part = 0; part < parts; ++part)
       for (int half = 0; half < 2; ++half)
         for (int m = 0; m < mb; ++m)
-          tma_load_2d(sbase + (part ? Smem::q_lo : Smem::q_hi) + half * kHalfBytesQ + m * 128 * 128, tm_q, bars.q_full(),
-                      half * 64, part * a.lo_row_offset + w.qrow_base + qg * kGroupRows + m * 128);
+          tma_load_2d(sbase + (part ? G::q_lo : G::q_hi) + half * G::kHalfBytesQ + m * 128 * 128, tm_q, bars.q_full(),
+                      half * 64, part * a.lo_row_offset + w.qrow_base + qg * G::kRows + m * 128);
     for (int ti = (qg == 0 ? n_first : 0); ti < w.nt; ++ti) {
       const int s = li % kStages;
       if (li >= kStages) ok = mbar_wait(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status);
