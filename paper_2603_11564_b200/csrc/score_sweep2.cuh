@@ -5,9 +5,8 @@
 // A job is one [128 keys x 256 queries] accumulator (two fit; four of 128 columns in the compact
 // geometry).  All four epilogue groups work
 // on every job, a quarter of the query columns each (sixteen epilogue warps, four per scheduler,
-// hide the latency of the tensor-memory loads and of the hand-offs); three groups hand their
-// partial sums to the fourth through consumed columns of the same accumulator (the groups take
-// that part in turn, job by job, so none of them lags behind), and that group's thread
+// hide the latency of the tensor-memory loads and of the hand-offs); groups 1-3 hand their
+// partial sums to group 0 through consumed columns of the same accumulator, and group 0's thread
 // (lane = key) stores the key's score: one coalesced fp32 per lane.  Before the first job the
 // epilogue threads merge the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the
 // resident query rows.
@@ -171,8 +170,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           }
         }
         float sum = (acc.x + acc.y) + (acc1.x + acc1.y);
-        const int red = job % kEpiGroups;                       // the group that sums this job's partials: each in turn
-        if (eg != red) {
+        if (eg > 0) {
           // hand the partial sum over in the first column this group has consumed (nothing to hand over
           // if it had no columns), then release the accumulator
           if (np > 0) {
@@ -186,16 +184,15 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job / kAcc) & 1, abort_flag, a.status));
           if (!ok) break;
           tc_fence_after();
-          // the other groups' partial sums: loads issued together, one wait (a group without columns left
-          // nothing); own slot and empty slots stay zero, the order of the additions is fixed
-          uint32_t part[kEpiGroups] = {0u, 0u, 0u, 0u};
+          // the three partial sums: loads issued together, one wait (a group without columns left nothing)
+          uint32_t part[kEpiGroups - 1] = {0u, 0u, 0u};
 #pragma unroll
-          for (int g = 0; g < kEpiGroups; ++g) {
+          for (int g = 1; g < kEpiGroups; ++g) {
             const int gp0 = (g * nch) / kEpiGroups, gnp = ((g + 1) * nch) / kEpiGroups - gp0;
-            if (g != eg && gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g]);
+            if (gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g - 1]);
           }
-          tmem_ld_wait4(part[0], part[1], part[2], part[3]);
-          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + (__uint_as_float(part[2]) + __uint_as_float(part[3]));
+          tmem_ld_wait3(part[0], part[1], part[2]);
+          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + __uint_as_float(part[2]);
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.acc_empty(buf));

@@ -14,8 +14,8 @@
 //   sweep 2 (score_sweep2.cuh)  keys on lanes, up to 256 query columns per MMA: merges the
 //             partials into each query's log-sum-exp, then sums exp2(s - lse_i) per key.
 // When the G*N rows of a KV head fit one block of 128 (N = 32 with G = 4) both sweeps run in a
-// compact geometry: half the shared memory for the queries, a deeper K ring, and four
-// accumulators of 128 columns in sweep 2.
+// compact geometry: half the shared memory for the queries, a third K stage in sweep 1, and
+// four accumulators of 128 columns in sweep 2.
 // The rotated queries are used as a bf16 pair (hi + lo, lo = bf16(q - hi)): two MMAs per
 // k-step with the same K tile.  A single bf16 rounding of q would put the per-token scores
 // of caches with outlier channels outside the 2e-3 tolerance.

@@ -17,8 +17,8 @@ constexpr int kStageBytes2 = kTile2 * 256, kHalfBytes2 = kTile2 * 128;
 
 // Geometry of a CTA.  kCompact = the G*N query rows of a KV head fit one block of 128 (the
 // paper's default window, N = 32 with four query heads per KV head): the query operand then
-// takes 64 KB instead of 128 KB, the K ring grows from 96 KB to 160 KB, and sweep 2 runs four
-// accumulators of 128 columns instead of two of 256.
+// takes 64 KB instead of 128 KB, sweep 1 (which streams K from DRAM) gets a third K stage, and
+// sweep 2 runs four accumulators of 128 columns instead of two of 256.
 template <bool kCompact>
 struct Geo {
   static constexpr int kRows = kCompact ? 128 : 256;          // query rows resident per group
@@ -26,7 +26,8 @@ struct Geo {
   static constexpr int kQBytes = 2 * kHalfBytesQ;             // per precision part (hi / lo)
   static constexpr int kRingBytes = 224 * 1024 - 2 * kQBytes;
   static constexpr int kStages1 = kRingBytes / kStageBytes1;  // 2 / 3 tiles of 192 keys
-  static constexpr int kStages2 = kRingBytes / kStageBytes2;  // 3 / 5 tiles of 128 keys
+  static constexpr int kStages2 = 3;                          // tiles of 128 keys (a deeper ring slows sweep 2 down:
+                                                              // its MMAs already take most of the shared-memory bandwidth)
   static constexpr int kAcc2 = kCompact ? 4 : 2;              // accumulators of sweep 2
   static constexpr int kAccCols2 = kTmemCols / kAcc2;
   // shared memory (offsets from the 1024-aligned base): query group as a bf16 pair, K ring
@@ -34,13 +35,13 @@ struct Geo {
   static constexpr int q_lo = kQBytes;
   static constexpr int k = 2 * kQBytes;
 };
-constexpr int kMaxStages = 5, kMaxAcc = 4;
+constexpr int kMaxStages = 3, kMaxAcc = 4;
 // ... followed, at the same place in both geometries, by the barriers, the group's log-sum-exp
 // (sweep 2) and two words.
 struct Smem {
   static constexpr int bars = 224 * 1024;
-  // barriers (24 x 8 B): k_full[5], k_empty[5], acc_full[4], acc_empty[4], q_full, q_empty, half_done[4]
-  static constexpr int lse = bars + 24 * 8;          // [256] floats
+  // barriers (20 x 8 B): k_full[3], k_empty[3], acc_full[4], acc_empty[4], q_full, q_empty, half_done[4]
+  static constexpr int lse = bars + 20 * 8;          // [256] floats
   static constexpr int tmem_ptr = lse + 256 * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
@@ -48,7 +49,7 @@ struct Smem {
 static_assert(Geo<false>::k + Geo<false>::kStages1 * kStageBytes1 <= Smem::bars && Geo<true>::k + Geo<true>::kStages1 * kStageBytes1 <= Smem::bars &&
               Geo<false>::k + Geo<false>::kStages2 * kStageBytes2 <= Smem::bars && Geo<true>::k + Geo<true>::kStages2 * kStageBytes2 <= Smem::bars,
               "K ring overruns the barriers");
-static_assert(Geo<true>::kStages2 <= kMaxStages && Geo<true>::kAcc2 <= kMaxAcc, "barrier table too small");
+static_assert(Geo<true>::kStages1 <= kMaxStages && Geo<true>::kStages2 <= kMaxStages && Geo<true>::kAcc2 <= kMaxAcc, "barrier table too small");
 constexpr int kSmemBytes = Smem::total + 1024;   // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
@@ -110,7 +111,7 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
     for (int i = 0; i < n_acc; ++i) {
       mbar_init(bars.acc_full(i), 1);
       mbar_init(bars.acc_empty(i), 4 * kEpiGroups);        // every epilogue warp reads every accumulator
-      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the three groups that hand their partial sums over
+      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the groups that hand their partial sums to group 0
     }
     mbar_init(bars.q_full(), 1);
     mbar_init(bars.q_empty(), 1);

@@ -179,12 +179,12 @@ __device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 512;
 __device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t v) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(v) : "memory");
 }
-// (issue only: tmem_ld_wait4 below completes up to four of these at once)
+// (issue only: tmem_ld_wait3 below completes up to three of these at once)
 __device__ __forceinline__ void tmem_ld1_issue(uint32_t taddr, uint32_t& v) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait4(uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(a), "+r"(b), "+r"(c), "+r"(d) :: "memory");
+__device__ __forceinline__ void tmem_ld_wait3(uint32_t& a, uint32_t& b, uint32_t& c) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(a), "+r"(b), "+r"(c) :: "memory");
 }
 // Descriptor of the operand `bytes` further on in shared memory (the start-address field is
 // in 16-byte units in the low bits and never carries out of it for addresses below 256 KB).
