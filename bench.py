@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
 
-One step = dapq_evict over every layer of the chosen configuration's synthetic cache
+One step = dapq_evict_layers over every layer of the chosen configuration's synthetic cache
 (default: the Llama-3-8B-shaped 32k-token cache).  The metric is prompt tokens scored and
 evicted per second per layer: tokens * layers / time.  Rank 0 prints one JSON line.
 
@@ -258,9 +258,12 @@ def run_ours(args, w: gi.Workload):
                        "v_out": torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt, device=dev)})
     torch.cuda.synchronize()
 
+    lq, lk, lv, lko, lvo = ([L[x] for L in layers] for x in ("q", "k", "v", "k_out", "v_out"))
+
     def step():
-        for L in layers:
-            dq.dapq_evict(ctx, L["q"], L["k"], L["v"], w.cu_rows, w.prompt_lens, w.keep, L["k_out"], L["v_out"])
+        # every layer in one call: the same kernels as one dapq_evict per layer, the rotation of layer l + 1
+        # running beside the selection and compaction of layer l
+        dq.dapq_evict_layers(ctx, lq, lk, lv, w.cu_rows, w.prompt_lens, w.keep, lko, lvo)
 
     def barrier():
         torch.cuda.synchronize()

@@ -375,7 +375,8 @@ dapq_status dapq_rope_pseudo_q(dapq_ctx* ctx, const void* q_pre, const int32_t* 
   dapq_status st = build_table(ctx, batch, nullptr, nullptr, nullptr, nullptr, pos_start_host, &t);
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
-  cudaError_t e = launch_rope(ctx->shape.dtype, ctx->shape.dtype, 0, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, (cudaStream_t)stream, &ctx->log);
+  cudaError_t e = launch_rope(ctx->shape.dtype, ctx->shape.dtype, 0, q_pre, q_rot, ctx->inv_freq, t, ctx->dims, false, (cudaStream_t)stream,
+                              &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
   return DAPQ_OK;
 }
@@ -446,9 +447,14 @@ dapq_status dapq_recall(dapq_ctx* ctx, const int32_t* idx_gold, const int32_t* i
   return DAPQ_OK;
 }
 
-dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
-                       const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
-                       float* scores_out, void* stream) {
+namespace {
+
+// after_own_compaction: the kernel before this call in `stream` is the compaction kernel of an
+// earlier evict on the same context (the layers of dapq_evict_layers); the rotation then does
+// not wait for it before it starts.
+dapq_status evict_impl(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache, const int32_t* k_keep_host,
+                       void* k_out, void* v_out, int32_t* idx_out, float* scores_out, void* stream,
+                       bool after_own_compaction) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
   if (!q_pre || !k_keep_host || !k_out || !v_out) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict: NULL argument");
   if (!aligned16(k_out) || !aligned16(v_out)) return fail(ctx, DAPQ_ERR_UNSUPPORTED, "k_out / v_out must be 16-byte aligned");
@@ -469,12 +475,13 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   if (wants_umma(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {
     // tensor-core scorer: rotated queries as a bf16 pair hi + lo (two MMAs per k-step)
     e = launch_rope(ctx->shape.dtype, kRopeOutSplitBf16, lo_rows * kHeadDim, q_pre, ctx->q_rot, ctx->inv_freq, t,
-                    ctx->dims, s, &ctx->log);
+                    ctx->dims, after_own_compaction, s, &ctx->log);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
     st = run_score_umma(ctx, plan, t, nullptr, scores, score_stride, nullptr, s);
   } else {
     // CUDA-core scorer: reads the rotated queries unrounded (fp32)
-    e = launch_rope(ctx->shape.dtype, kRopeOutF32, 0, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, s, &ctx->log);
+    e = launch_rope(ctx->shape.dtype, kRopeOutF32, 0, q_pre, ctx->q_rot, ctx->inv_freq, t, ctx->dims, after_own_compaction, s,
+                    &ctx->log);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
     st = run_score(ctx, DAPQ_F32, ctx->q_rot, cd, t, nullptr, scores, score_stride, nullptr, nullptr, s);
   }
@@ -486,6 +493,14 @@ dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   return DAPQ_OK;
 }
 
+}  // namespace
+
+dapq_status dapq_evict(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* cache,
+                       const int32_t* k_keep_host, void* k_out, void* v_out, int32_t* idx_out,
+                       float* scores_out, void* stream) {
+  return evict_impl(ctx, q_pre, cache, k_keep_host, k_out, v_out, idx_out, scores_out, stream, false);
+}
+
 dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre,
                               const dapq_cache_view* caches, const int32_t* k_keep_host,
                               int64_t k_keep_layer_stride, void* const* k_out, void* const* v_out,
@@ -495,8 +510,8 @@ dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const void* const
   if (n_layers > 0 && (!q_pre || !caches || !k_keep_host || !k_out || !v_out))
     return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers: NULL argument");
   for (int32_t l = 0; l < n_layers; ++l) {
-    const dapq_status st = dapq_evict(ctx, q_pre[l], &caches[l], k_keep_host + (int64_t)l * k_keep_layer_stride, k_out[l],
-                                      v_out[l], idx_out ? idx_out[l] : nullptr, nullptr, stream);
+    const dapq_status st = evict_impl(ctx, q_pre[l], &caches[l], k_keep_host + (int64_t)l * k_keep_layer_stride, k_out[l],
+                                      v_out[l], idx_out ? idx_out[l] : nullptr, nullptr, stream, l > 0);
     if (st != DAPQ_OK) return st;
   }
   return DAPQ_OK;

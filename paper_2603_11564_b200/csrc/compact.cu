@@ -14,6 +14,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 compact_kv_kernel(const CacheDev cv, int elem_bytes, const int32_t* __restrict__ idx, int64_t idx_stride,
                   uint4* __restrict__ k_out, uint4* __restrict__ v_out,
                   const __grid_constant__ SeqTable t, int* __restrict__ status) {
+  pdl_trigger();                     // whatever follows may be set up (or, if it does not depend on this copy, run) beside it
   pdl_wait();
   const int kt = t.cu_keep[t.batch];
   const int64_t gid = (int64_t)blockIdx.x * kCompactThreads + threadIdx.x;

@@ -84,7 +84,10 @@ struct LaunchLog {
 // while the predecessor still runs.  The short kernels that precede a long one (rotation,
 // selection) also signal at their start that the next kernel may be scheduled (pdl_trigger); the
 // sweeps do not: their successors' CTAs would only sit on the SMs the next sweep needs (measured:
-// slower).  Both are no-ops for a kernel launched the ordinary way.
+// slower).  The compaction signals at its start too: in dapq_evict_layers the next layer's
+// rotation, which touches nothing the compaction or the selection before it use, runs beside
+// them and waits at its END, so that the kernels after it stay ordered behind the compaction.
+// Both instructions are no-ops for a kernel launched the ordinary way.
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -119,7 +122,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 // the CUDA-core scorer) or a bf16 pair hi + lo with lo = bf16(q - hi) stored `lo_offset`
 // elements after hi (for the tensor-core scorer).
 cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* q_pre, void* q_rot, const double* inv_freq_dev,
-                        const SeqTable& t, const Dims& dm, cudaStream_t s, LaunchLog* log);
+                        const SeqTable& t, const Dims& dm, bool late_wait, cudaStream_t s, LaunchLog* log);
 
 // Generic CUDA-core scorer (any N <= 128, both dtypes).
 //   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits, room for max_chunks

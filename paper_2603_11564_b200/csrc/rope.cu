@@ -31,12 +31,18 @@ template <typename T, typename TO, bool kSplit>
 __global__ void __launch_bounds__(kHeadDim / 2 * kHeadsPerBlock)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
-                     int n_q_heads, int n_pseudo, int64_t lo_offset) {
+                     int n_q_heads, int n_pseudo, int64_t lo_offset, int late_wait) {
+  // late_wait: the kernel before this one in the stream neither writes q_pre nor still reads q_rot
+  // (it is the compaction of the layer before), so the rotation runs beside it; the wait at the end
+  // keeps this grid, and with it everything launched after it, ordered behind that kernel.
   pdl_trigger();
-  pdl_wait();
+  if (!late_wait) pdl_wait();
   const int i = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const int h = blockIdx.z * kHeadsPerBlock + threadIdx.y;
-  if (h >= n_q_heads) return;
+  if (h >= n_q_heads) {
+    if (late_wait) pdl_wait();
+    return;
+  }
   constexpr int half = kHeadDim / 2;
   const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
   const double lo = to_double<T>(q_pre[base + c]);
@@ -52,28 +58,30 @@ rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
     q_rot[lo_offset + base + c] = from_double<TO>(r0 - to_double<TO>(h0));
     q_rot[lo_offset + base + c + half] = from_double<TO>(r1 - to_double<TO>(h1));
   }
+  if (late_wait) pdl_wait();
 }
 
 }  // namespace
 
 cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* q_pre, void* q_rot,
-                        const double* inv_freq_dev, const SeqTable& t, const Dims& dm, cudaStream_t s,
-                        LaunchLog* log) {
+                        const double* inv_freq_dev, const SeqTable& t, const Dims& dm, bool late_wait,
+                        cudaStream_t s, LaunchLog* log) {
+  const int lw = late_wait ? 1 : 0;
   log->begin(kKindRope, s);
   dim3 grid(dm.n_pseudo, t.batch, (dm.n_q_heads + kHeadsPerBlock - 1) / kHeadsPerBlock);
   dim3 block(kHeadDim / 2, kHeadsPerBlock);
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
   } else if (dtype == DAPQ_BF16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, float, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
   } else {
     launch_pdl(rope_pseudo_q_kernel<float, float, false>, grid, block, 0, s, 1, (const float*)q_pre, (float*)q_rot,
-               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0);
+               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
   }
   log->end(s);
   return cudaGetLastError();
