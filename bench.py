@@ -45,8 +45,11 @@ FALLBACK_BF16_TFLOPS = 1590.0
 NCU_TRAFFIC_BYTES = {
     # profiles/evict_kernels_llama3_8b_32k.md (a 2-layer run of the same command; traffic per launch does not
     # depend on the number of layers)
-    ("sweep1", "llama3_8b_32k"): 68331264 + 693504,
-    ("sweep2", "llama3_8b_32k"): 69376768 + 887040,
+    ("sweep1", "llama3_8b_32k"): 68331520 + 467712,
+    ("sweep2", "llama3_8b_32k"): 69376256 + 606464,
+    # profiles/evict_kernels_batched_serving.md
+    ("sweep1", "batched_serving"): 315072000 + 6724352,
+    ("sweep2", "batched_serving"): 314087936 + 6920704,
 }
 
 
