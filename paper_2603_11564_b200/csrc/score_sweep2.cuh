@@ -104,12 +104,12 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * kEpiGroups * rows_pad + grow;
             const int64_t step = (int64_t)a.n_kv_heads * kEpiGroups * rows_pad;
             const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
-            // one pass, eight independent loads in flight; (max, sum) merged in chunk order
+            // one pass, sixteen independent loads in flight; (max, sum) merged in chunk order
             float mx = -CUDART_INF_F, z = 0.f;
-            for (int c0 = 0; c0 < nc; c0 += 2) {
-              float2 q[8];
+            for (int c0 = 0; c0 < nc; c0 += 4) {
+              float2 q[16];
 #pragma unroll
-              for (int u = 0; u < 2; ++u) {
+              for (int u = 0; u < 4; ++u) {
                 const bool in = c0 + u < nc;
 #pragma unroll
                 for (int g = 0; g < kEpiGroups; ++g)
@@ -117,13 +117,13 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
               }
               float m8 = q[0].x;
 #pragma unroll
-              for (int u = 1; u < 8; ++u) m8 = fmaxf(m8, q[u].x);
+              for (int u = 1; u < 16; ++u) m8 = fmaxf(m8, q[u].x);
               if (m8 > mx) {
                 z *= exp2f(mx - m8);                        // exp2f(-inf) = 0 on the first chunk
                 mx = m8;
               }
 #pragma unroll
-              for (int u = 0; u < 8; ++u) z += q[u].y * exp2f(q[u].x - mx);
+              for (int u = 0; u < 16; ++u) z += q[u].y * exp2f(q[u].x - mx);
             }
             l2 = mx + log2f(z);
           }

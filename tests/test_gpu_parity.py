@@ -540,3 +540,29 @@ def test_prompt_window_variant_uses_the_same_entry_points(dq):
         kept = np.concatenate([idx[h].cpu().numpy(), np.arange(L - N, L)])      # the caller appends the window rows
         assert len(np.unique(kept)) == keep
     dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------------------------- seeded random shapes, end to end
+def _random_cases(n_cases, seed=20260311):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n_cases):
+        hkv = int(rng.choice([1, 2, 4, 8]))
+        group = int(rng.choice([1, 2, 4, 7, 8]))
+        n = int(rng.choice([1, 3, 16, 17, 32, 33, 64, 100, 128]))
+        batch = int(rng.integers(1, 5))
+        lens = tuple(int(x) for x in np.maximum(1, (rng.pareto(1.2, batch) * 150).astype(np.int64) % 2600 + rng.integers(1, 40, batch)))
+        keep = tuple(int(rng.integers(1, L + 1)) for L in lens)
+        dtype = "bf16" if rng.random() < 0.75 else "f32"
+        cases.append((dtype, hkv * group, hkv, n, lens, keep))
+    return cases
+
+
+@pytest.mark.parametrize("dtype,hq,hkv,n,lens,keep", _random_cases(16))
+def test_evict_random_shapes(dq, dtype, hq, hkv, n, lens, keep):
+    """Seeded random head counts, window sizes, ragged batches and budgets through the whole path (both
+    scorers, both geometries of the tensor-core sweeps, every top-k cluster size that these lengths reach)."""
+    w = _small(lens=lens, keep=keep, dtype=dtype, n_q_heads=hq, n_kv_heads=hkv, n_pseudo=n, n_needles=0,
+               outlier_channels=2 if dtype == "bf16" else 0)
+    data = gi.draw_layer(w, 0, "cpu")
+    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
