@@ -33,12 +33,14 @@ def rope_inv_freq(head_dim: int, rope_base: float) -> np.ndarray:
 
 
 def rope_pseudo_q(q_pre: np.ndarray, pos_start: int, rope_base: float,
-                  inv_freq: Optional[np.ndarray] = None) -> np.ndarray:
+                  inv_freq: Optional[np.ndarray] = None, interleaved: bool = False) -> np.ndarray:
     """Rotate pseudo queries to positions pos_start + i (Section 4.1, position assignment).
 
     q_pre [..., N, d].  Rotate-half pairing: channel c is paired with channel c + d/2,
       out[c]       = q[c]     cos(p theta_c) - q[c+d/2] sin(p theta_c)
       out[c + d/2] = q[c+d/2] cos(p theta_c) + q[c]     sin(p theta_c).
+    interleaved: the pair of frequency c is (2c, 2c + 1) instead (the paper only says "RoPE";
+    rotate-half is what its Llama / Qwen models use, adjacent pairs the other common layout).
     """
     q = np.asarray(q_pre, dtype=np.float64)
     n, d = q.shape[-2], q.shape[-1]
@@ -47,8 +49,13 @@ def rope_pseudo_q(q_pre: np.ndarray, pos_start: int, rope_base: float,
     pos = np.float64(pos_start) + np.arange(n, dtype=np.float64)
     ang = pos[:, None] * theta[None, :]                    # [N, d/2]
     cos, sin = np.cos(ang), np.sin(ang)
-    lo, hi = q[..., :half], q[..., half:]
     out = np.empty_like(q)
+    if interleaved:
+        lo, hi = q[..., 0::2], q[..., 1::2]
+        out[..., 0::2] = lo * cos - hi * sin
+        out[..., 1::2] = hi * cos + lo * sin
+        return out
+    lo, hi = q[..., :half], q[..., half:]
     out[..., :half] = lo * cos - hi * sin
     out[..., half:] = hi * cos + lo * sin
     return out
@@ -185,7 +192,8 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
           prompt_len: Sequence[int], k_keep: Sequence[int], rope_base: float,
           scale: Optional[float] = None,
           pos_start: Optional[Sequence[int]] = None, pool_mode: str = "none",
-          pool_kernel: int = 1, inv_freq: Optional[np.ndarray] = None) -> Dict[str, object]:
+          pool_kernel: int = 1, inv_freq: Optional[np.ndarray] = None,
+          rope_interleaved: bool = False) -> Dict[str, object]:
     """The whole path for one layer (Figure 1): rotate, score, select, compact.
 
     q_pre [B, H_q, N, d] pre-RoPE pseudo queries (any float dtype; converted exactly
@@ -208,7 +216,7 @@ def evict(q_pre: np.ndarray, k: np.ndarray, v: np.ndarray, cu_rows: Sequence[int
         r0 = int(cu_rows[b])
         assert int(cu_rows[b + 1]) - r0 == L + n
         p0 = L if pos_start is None else int(pos_start[b])
-        q_rot = rope_pseudo_q(np.asarray(q_pre[b], dtype=np.float64), p0, rope_base, inv_freq)
+        q_rot = rope_pseudo_q(np.asarray(q_pre[b], dtype=np.float64), p0, rope_base, inv_freq, rope_interleaved)
         k_seq = k[:, r0:r0 + L + n]
         v_seq = v[:, r0:r0 + L + n]
         res = score_sequence(q_rot, k_seq, L, G, scale)

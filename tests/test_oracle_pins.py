@@ -65,6 +65,26 @@ def test_rope_identity_norm_and_relative_property():
         np.testing.assert_allclose(a, b, atol=1e-9)
 
 
+def test_rope_interleaved_pairs_hand_case_and_library():
+    # Adjacent pairs: (1,2) by 90 degrees -> (-2,1); (3,4) by 180 degrees -> (-3,-4).
+    q = np.array([[1.0, 2.0, 3.0, 4.0]])
+    out = orc.rope_pseudo_q(q, pos_start=1, rope_base=1.0, inv_freq=np.array([math.pi / 2, math.pi]),
+                            interleaved=True)
+    np.testing.assert_allclose(out, [[-2.0, 1.0, -3.0, -4.0]], atol=1e-14)
+    # As complex numbers x[2c] + i x[2c+1], the rotation is a multiplication by exp(i p theta_c).
+    q = _rand((2, 7, 16), 11)
+    z = torch.view_as_complex(torch.from_numpy(q).reshape(2, 7, 8, 2).contiguous())
+    theta = torch.from_numpy(orc.rope_inv_freq(16, 1.0e4))
+    pos = torch.arange(300, 307, dtype=torch.float64)
+    rot = torch.polar(torch.ones(7, 8, dtype=torch.float64), pos[:, None] * theta[None, :])
+    want = torch.view_as_real(z * rot).reshape(2, 7, 16).numpy()
+    np.testing.assert_allclose(orc.rope_pseudo_q(q, 300, 1.0e4, interleaved=True), want, atol=1e-12)
+    # and it is the rotate-half form seen through the channel permutation 2c -> c, 2c + 1 -> c + d/2
+    perm = np.concatenate([np.arange(0, 16, 2), np.arange(1, 16, 2)])
+    half = orc.rope_pseudo_q(q[..., perm], 300, 1.0e4)
+    np.testing.assert_allclose(orc.rope_pseudo_q(q, 300, 1.0e4, interleaved=True)[..., perm], half, atol=1e-13)
+
+
 def test_rope_angle_precision_at_128k():
     # double-precision angles at the largest position used (131072 + 127) agree with
     # extended precision to far below the scorer's tolerance
