@@ -77,8 +77,11 @@ enum { DAPQ_MAX_BATCH = 128, DAPQ_MAX_PSEUDO = 128, DAPQ_HEAD_DIM = 128, DAPQ_MA
 typedef enum { DAPQ_POOL_NONE = 0, DAPQ_POOL_MAX = 1, DAPQ_POOL_AVG = 2 } dapq_pool_mode;
 
 /* dapq_shape.flags.  DAPQ_FLAG_CUDA_CORE_SCORER keeps the scorer on the CUDA-core kernels
- * (fp32 arithmetic on unrounded rotated queries) even where the tensor-core path applies. */
-typedef enum { DAPQ_FLAG_CUDA_CORE_SCORER = 1 } dapq_flags;
+ * (fp32 arithmetic on unrounded rotated queries) even where the tensor-core path applies.
+ * DAPQ_FLAG_ROPE_INTERLEAVED: the rotation pairs channel 2c with 2c + 1 instead of c with
+ * c + d/2 (Section 4.1 only says "RoPE"; the rotate-half pairing of the paper's Llama and Qwen
+ * models is the default; the cache's keys must have been rotated with the same pairing). */
+typedef enum { DAPQ_FLAG_CUDA_CORE_SCORER = 1, DAPQ_FLAG_ROPE_INTERLEAVED = 2 } dapq_flags;
 
 typedef struct dapq_ctx dapq_ctx;
 

@@ -22,6 +22,7 @@ DAPQ_OK, DAPQ_ERR_INVALID_ARG, DAPQ_ERR_UNSUPPORTED, DAPQ_ERR_WORKSPACE, DAPQ_ER
 DAPQ_BF16, DAPQ_F32 = 0, 1
 DAPQ_POOL_NONE, DAPQ_POOL_MAX, DAPQ_POOL_AVG = 0, 1, 2
 DAPQ_FLAG_CUDA_CORE_SCORER = 1
+DAPQ_FLAG_ROPE_INTERLEAVED = 2
 _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORTED",
                  3: "DAPQ_ERR_WORKSPACE", 4: "DAPQ_ERR_CUDA", 5: "DAPQ_ERR_TIMEOUT"}
 

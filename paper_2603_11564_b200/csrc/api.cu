@@ -252,7 +252,7 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   if (sh->max_batch > kMaxBatch || sh->max_total_rows > 0x7fffffffLL)
     return bail(DAPQ_ERR_UNSUPPORTED, "max_batch > 128 or max_total_rows >= 2^31");
   if (sh->dtype != DAPQ_BF16 && sh->dtype != DAPQ_F32) return bail(DAPQ_ERR_INVALID_ARG, "unknown dtype");
-  if (sh->flags & ~DAPQ_FLAG_CUDA_CORE_SCORER) return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
+  if (sh->flags & ~(DAPQ_FLAG_CUDA_CORE_SCORER | DAPQ_FLAG_ROPE_INTERLEAVED)) return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
   if (sh->pool_mode != DAPQ_POOL_NONE && sh->pool_mode != DAPQ_POOL_MAX && sh->pool_mode != DAPQ_POOL_AVG)
     return bail(DAPQ_ERR_INVALID_ARG, "unknown pool_mode");
   if (sh->pool_mode != DAPQ_POOL_NONE && (sh->pool_kernel < 3 || sh->pool_kernel > DAPQ_MAX_POOL_KERNEL || sh->pool_kernel % 2 == 0))
@@ -268,6 +268,7 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   ctx->dims.n_kv_heads = sh->n_kv_heads;
   ctx->dims.group = sh->n_q_heads / sh->n_kv_heads;
   ctx->dims.n_pseudo = sh->n_pseudo;
+  ctx->dims.rope_interleaved = (sh->flags & DAPQ_FLAG_ROPE_INTERLEAVED) ? 1 : 0;
   const double scale = sh->softmax_scale > 0.f ? (double)sh->softmax_scale : 1.0 / sqrt((double)kHeadDim);
   ctx->dims.scale_log2e = (float)(scale * 1.4426950408889634074);
 

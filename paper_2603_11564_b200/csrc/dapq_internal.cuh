@@ -45,6 +45,7 @@ struct CacheDev {
 struct Dims {
   int32_t n_q_heads, n_kv_heads, group, n_pseudo;
   float scale_log2e;                // softmax scale * log2(e): logits are kept in base 2
+  int32_t rope_interleaved = 0;     // RoPE pairs are (2c, 2c + 1) instead of (c, c + d/2)
 };
 
 // Device status word bits (set by kernels, read by dapq_poll_status).

@@ -3,7 +3,7 @@
 // the first N decoding steps).
 //
 // Grid (pseudo query i, sequence b, block of query heads); thread (c, hy) owns the channel
-// pair (c, c + d/2) of one head.  The angle pos * theta_c is formed and reduced in double
+// pair of frequency c of one head: (c, c + d/2), or (2c, 2c + 1) for the interleaved layout.  The angle pos * theta_c is formed and reduced in double
 // precision: at positions near 131k a float angle has only ~7 fractional bits, which alone
 // would cost half of the scorer's error budget.  Each thread evaluates its own sincos (the
 // table is tiny: B*N*64 angles), so no thread waits on another and the launch is one short
@@ -31,7 +31,8 @@ template <typename T, typename TO, bool kSplit>
 __global__ void __launch_bounds__(kHeadDim / 2 * kHeadsPerBlock)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
-                     int n_q_heads, int n_pseudo, int64_t lo_offset, int late_wait) {
+                     int n_q_heads, int n_pseudo, int64_t lo_offset, int late_wait,
+                     int interleaved) {
   // late_wait: the kernel before this one in the stream neither writes q_pre nor still reads q_rot
   // (it is the compaction of the layer before), so the rotation runs beside it; the wait at the end
   // keeps this grid, and with it everything launched after it, ordered behind that kernel.
@@ -45,18 +46,19 @@ rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
   }
   constexpr int half = kHeadDim / 2;
   const size_t base = (((size_t)b * n_q_heads + h) * n_pseudo + i) * kHeadDim;
-  const double lo = to_double<T>(q_pre[base + c]);
-  const double hi = to_double<T>(q_pre[base + c + half]);
+  const size_t e0 = base + (interleaved ? 2 * c : c), e1 = interleaved ? e0 + 1 : e0 + half;
+  const double lo = to_double<T>(q_pre[e0]);
+  const double hi = to_double<T>(q_pre[e1]);
   const double ang = (double)(t.pos_start[b] + i) * inv_freq[c];
   double sn, cs;
   sincos(ang, &sn, &cs);
   const double r0 = lo * cs - hi * sn, r1 = hi * cs + lo * sn;
   const TO h0 = from_double<TO>(r0), h1 = from_double<TO>(r1);
-  q_rot[base + c] = h0;
-  q_rot[base + c + half] = h1;
+  q_rot[e0] = h0;
+  q_rot[e1] = h1;
   if (kSplit) {
-    q_rot[lo_offset + base + c] = from_double<TO>(r0 - to_double<TO>(h0));
-    q_rot[lo_offset + base + c + half] = from_double<TO>(r1 - to_double<TO>(h1));
+    q_rot[lo_offset + e0] = from_double<TO>(r0 - to_double<TO>(h0));
+    q_rot[lo_offset + e1] = from_double<TO>(r1 - to_double<TO>(h1));
   }
   if (late_wait) pdl_wait();
 }
@@ -72,16 +74,16 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
   dim3 block(kHeadDim / 2, kHeadsPerBlock);
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw, dm.rope_interleaved);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
   } else if (dtype == DAPQ_BF16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, float, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
+               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
   } else {
     launch_pdl(rope_pseudo_q_kernel<float, float, false>, grid, block, 0, s, 1, (const float*)q_pre, (float*)q_rot,
-               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw);
+               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
   }
   log->end(s);
   return cudaGetLastError();

@@ -43,7 +43,7 @@ def test_struct_layouts_match_the_header(lib):
     (dict(head_dim=64), 2), (dict(n_pseudo=129), 2), (dict(n_pseudo=0), 2), (dict(n_kv_heads=3), 1),
     (dict(max_batch=0), 1), (dict(max_batch=129), 2), (dict(dtype=7), 1), (dict(rope_base=0.0), 1),
     (dict(softmax_scale=-1.0), 1), (dict(max_total_rows=0), 1), (dict(pool_mode=5), 1),
-    (dict(pool_mode=1, pool_kernel=4), 2), (dict(pool_mode=2, pool_kernel=129), 2),
+    (dict(pool_mode=1, pool_kernel=4), 2), (dict(pool_mode=2, pool_kernel=129), 2), (dict(flags=4), 1),
 ])
 def test_create_rejects_bad_shapes_without_a_device(lib, kw, status):
     args = dict(n_q_heads=8, n_kv_heads=2, n_pseudo=32, max_batch=1, max_total_rows=1000, dtype=0, rope_base=1e4)

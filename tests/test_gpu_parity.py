@@ -68,17 +68,19 @@ def _check_evict(w, data, got, ref):
 
 
 # ------------------------------------------------------------------------- dapq_rope_pseudo_q
+@pytest.mark.parametrize("interleaved", [False, True])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_rope_parity(dq, dtype):
+def test_rope_parity(dq, dtype, interleaved):
     w = _small(lens=(5, 131072, 4097), keep=(1, 1, 1), dtype=dtype, n_pseudo=33, rope_base=5.0e5, n_needles=0)
-    ctx = _ctx(dq, w)
+    ctx = _ctx(dq, w, flags=dq.DAPQ_FLAG_ROPE_INTERLEAVED if interleaved else 0)
     data = gi.draw_layer(dataclasses.replace(w, prompt_lens=(8, 8, 8)), 0, "cpu")
     q = data["q_pre"].cuda()
     out = torch.empty_like(q)
     pos = [5, 131072, 0]
     dq.dapq_rope_pseudo_q(ctx, q, pos, out)
     torch.cuda.synchronize()
-    ref = np.stack([orc.rope_pseudo_q(util.to_f64(data["q_pre"][b]), pos[b], w.rope_base) for b in range(3)])
+    ref = np.stack([orc.rope_pseudo_q(util.to_f64(data["q_pre"][b]), pos[b], w.rope_base, interleaved=interleaved)
+                    for b in range(3)])
     got = util.to_f64(out)
     tol = 2.0 ** -8 if dtype == "bf16" else 2.0 ** -22
     assert np.all(np.abs(got - ref) <= tol * np.abs(ref) + 1e-7)
@@ -417,6 +419,19 @@ def test_evict_with_scaled_rope_frequencies(dq):
     ctx = _ctx(dq, w, inv_freq=list(inv))
     _check_evict(w, data, _gpu_evict(dq, w, data, ctx), ref)
     dq.dapq_destroy(ctx)
+
+
+def test_evict_with_interleaved_rope_pairs(dq):
+    """DAPQ_FLAG_ROPE_INTERLEAVED through the whole path, on the tensor cores and on the CUDA cores."""
+    w = _small(lens=(800, 77), keep=(60, 9), n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    ref = orc.evict(util.to_f64(data["q_pre"]), util.to_f64(data["k"]), util.to_f64(data["v"]), w.cu_rows,
+                    w.prompt_lens, w.keep, w.rope_base, rope_interleaved=True)
+    assert not np.allclose(ref["scores"][0], util.oracle_evict(w, data)["scores"][0], rtol=1e-3)   # the pairing matters
+    for extra in (0, dq.DAPQ_FLAG_CUDA_CORE_SCORER):
+        ctx = _ctx(dq, w, flags=dq.DAPQ_FLAG_ROPE_INTERLEAVED | extra)
+        _check_evict(w, data, _gpu_evict(dq, w, data, ctx), ref)
+        dq.dapq_destroy(ctx)
 
 
 def test_shifted_positions_through_rope_and_score(dq):
