@@ -208,9 +208,12 @@ DAPQ_API dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const vo
 
 /* dapq_evict for callers whose tensors live in host memory: q_pre, the cache view's k / v
  * and k_out / v_out / idx_out are HOST pointers (pinned memory gives full copy speed).
- * Copies the inputs to device staging buffers owned by the context (allocated on first
+ * Copies q_pre and K to device staging buffers owned by the context (allocated on first
  * use, sized from dapq_shape), runs dapq_evict, copies the results back and synchronises
- * `stream` before returning. */
+ * `stream` before returning.  Of V only the retained rows are needed: when the caller's V is
+ * page-locked memory that the device can address (cudaHostAlloc, cudaHostRegister), the
+ * compaction kernel reads those rows from it directly and V is never copied as a whole;
+ * pageable V is staged like K. */
 DAPQ_API dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
                             const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
                             int32_t* idx_out_host, void* stream);

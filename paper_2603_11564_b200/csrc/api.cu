@@ -544,15 +544,29 @@ dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_ca
     DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_vo, cache_bytes));
     DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_idx, (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * sizeof(int32_t)));
   }
+  // Only the kept rows of V are needed.  If the caller's V is page-locked host memory that the device can
+  // address, the compaction kernel gathers those rows straight from it; otherwise V is staged like K.
+  const void* v_mapped = nullptr;
+  {
+    cudaPointerAttributes pa;
+    const int per16 = 16 / ctx->elem_bytes;                        // (the kernel reads 16-byte pieces)
+    const bool vector_ok = hv.v_row_stride % per16 == 0 && hv.v_head_stride % per16 == 0;
+    if (vector_ok && cudaPointerGetAttributes(&pa, hv.v) == cudaSuccess && pa.type == cudaMemoryTypeHost &&
+        pa.devicePointer && aligned16(pa.devicePointer))
+      v_mapped = pa.devicePointer;
+    else
+      cudaGetLastError();
+  }
   // device copy of the used row range [cu_rows[0], cu_rows[B]) of every head, packed from row 0
   const int64_t row0 = t.cu_rows[0], n_rows = t.cu_rows[t.batch] - row0;
   DAPQ_CUDA(ctx, cudaMemcpyAsync(ctx->h_q, q_pre_host, (size_t)t.batch * sh.n_q_heads * sh.n_pseudo * row_bytes,
                                  cudaMemcpyHostToDevice, s));
   for (int h = 0; h < sh.n_kv_heads; ++h) {
     const char* ks = (const char*)hv.k + ((size_t)h * hv.k_head_stride + (size_t)row0 * hv.k_row_stride) * eb;
-    const char* vs = (const char*)hv.v + ((size_t)h * hv.v_head_stride + (size_t)row0 * hv.v_row_stride) * eb;
     DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_k + (size_t)h * n_rows * row_bytes, row_bytes, ks,
                                      (size_t)hv.k_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
+    if (v_mapped) continue;
+    const char* vs = (const char*)hv.v + ((size_t)h * hv.v_head_stride + (size_t)row0 * hv.v_row_stride) * eb;
     DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_v + (size_t)h * n_rows * row_bytes, row_bytes, vs,
                                      (size_t)hv.v_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
   }
@@ -561,9 +575,17 @@ dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_ca
   dapq_cache_view dv;
   memset(&dv, 0, sizeof(dv));
   dv.k = ctx->h_k;
-  dv.v = ctx->h_v;
-  dv.k_head_stride = dv.v_head_stride = n_rows * kHeadDim;
-  dv.k_row_stride = dv.v_row_stride = kHeadDim;
+  dv.k_head_stride = n_rows * kHeadDim;
+  dv.k_row_stride = kHeadDim;
+  if (v_mapped) {
+    dv.v = (const char*)v_mapped + (size_t)row0 * hv.v_row_stride * eb;     // row 0 of the view = row cu_rows[0] of the caller's
+    dv.v_head_stride = hv.v_head_stride;
+    dv.v_row_stride = hv.v_row_stride;
+  } else {
+    dv.v = ctx->h_v;
+    dv.v_head_stride = n_rows * kHeadDim;
+    dv.v_row_stride = kHeadDim;
+  }
   dv.cu_rows_host = cu_local;
   dv.prompt_len_host = cache_host->prompt_len_host;
   dv.batch = t.batch;

@@ -267,13 +267,16 @@ def test_evict_edge_shapes(dq):
     np.testing.assert_array_equal(got["idx"][0, 1:65], np.arange(64))
 
 
-def test_evict_host_matches_device_call(dq):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_evict_host_matches_device_call(dq, pinned):
+    """Host buffers in, host buffers out.  Pinned V is gathered by the compaction kernel straight from host
+    memory; pageable V is staged on the device first."""
     w = gi.scaled_down("batched_serving", 32, n_layers=1)
     data = util.make_case(w)
     ctx = _ctx(dq, w)
     dev = _gpu_evict(dq, w, data, ctx)
     KT = int(w.cu_keep[-1])
-    pin = lambda t: t.contiguous().pin_memory()
+    pin = (lambda t: t.contiguous().pin_memory()) if pinned else (lambda t: t.contiguous().clone())
     k_out = torch.empty((w.n_kv_heads, KT, 128), dtype=torch.bfloat16).pin_memory()
     v_out = torch.empty_like(k_out).pin_memory()
     idx = torch.empty((w.n_kv_heads, KT), dtype=torch.int32).pin_memory()
