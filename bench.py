@@ -356,11 +356,12 @@ def run_ours(args, w: gi.Workload):
             host[-1]["v_out"] = torch.empty((w.n_kv_heads, KT, w.head_dim), dtype=dt).pin_memory()
             host[-1]["idx"] = torch.empty((w.n_kv_heads, KT), dtype=torch.int32).pin_memory()
 
+        hl = [host[l % n_host] for l in range(n_layers)]
+        hq, hk, hv, hko, hvo, hidx = ([H[x] for H in hl] for x in ("q", "k", "v", "k_out", "v_out", "idx"))
+
         def host_step():
-            for l in range(n_layers):
-                H = host[l % n_host]
-                dq.dapq_evict_host(ctx, H["q"], H["k"], H["v"], w.cu_rows, w.prompt_lens, w.keep,
-                                   H["k_out"], H["v_out"], H["idx"])
+            # every layer in one call: the copies of layer l + 1 run beside the kernels of layer l
+            dq.dapq_evict_layers_host(ctx, hq, hk, hv, w.cu_rows, w.prompt_lens, w.keep, hko, hvo, hidx)
 
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
         host_step()
@@ -380,7 +381,7 @@ def run_ours(args, w: gi.Workload):
         d2h = n_layers * (2 * w.n_kv_heads * KT * w.head_dim * eb + 4 * w.n_kv_heads * KT)
         e2e = {"value": whole_job_value(world, tokens, n_layers, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": e2e_steps,
-               "api": "dapq_evict_host (pinned host q/K/V in: q and K copied, kept V rows gathered over PCIe; compacted K/V + indices out, per layer)"}
+               "api": "dapq_evict_layers_host (pinned host q/K/V in: q and K copied, kept V rows gathered over PCIe; compacted K/V + indices out; copies of layer l+1 beside the kernels of layer l)"}
 
     dq.dapq_destroy(ctx)
 

@@ -218,6 +218,15 @@ DAPQ_API dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, cons
                             const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
                             int32_t* idx_out_host, void* stream);
 
+/* dapq_evict_host for every layer of a model (arguments as in dapq_evict_layers, all data
+ * pointers HOST pointers).  Two staging sets and a copy stream owned by the context let the
+ * host-to-device copies of layer l + 1 run beside the kernels and the device-to-host copies of
+ * layer l; the call returns after `stream` has been synchronised.  Not capturable into a graph. */
+DAPQ_API dapq_status dapq_evict_layers_host(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre_host,
+                                   const dapq_cache_view* caches_host, const int32_t* k_keep_host,
+                                   int64_t k_keep_layer_stride, void* const* k_out_host,
+                                   void* const* v_out_host, int32_t* const* idx_out_host, void* stream);
+
 /* The paper has no counterpart to this entry point; it exists for callers that may not
  * allocate device memory at the point where they need scores: engines whose own allocator owns
  * the whole device, plug-ins running after a "no more driver allocations" point, code between a

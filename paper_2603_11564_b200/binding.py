@@ -28,7 +28,7 @@ _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORT
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
            "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
-           "dapq_compact_kv", "dapq_evict", "dapq_evict_layers", "dapq_evict_host", "dapq_score_static", "dapq_recall")
+           "dapq_compact_kv", "dapq_evict", "dapq_evict_layers", "dapq_evict_host", "dapq_evict_layers_host", "dapq_score_static", "dapq_recall")
 
 
 class DapqError(RuntimeError):
@@ -92,6 +92,8 @@ def load_library() -> C.CDLL:
     lib.dapq_evict_layers.argtypes = [vp, C.c_int32, C.POINTER(vp), C.POINTER(dapq_cache_view), i32p, C.c_int64,
                                       C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
     lib.dapq_evict_layers.restype = C.c_int
+    lib.dapq_evict_layers_host.argtypes = lib.dapq_evict_layers.argtypes
+    lib.dapq_evict_layers_host.restype = C.c_int
     lib.dapq_evict_host.argtypes = [vp, vp, C.POINTER(dapq_cache_view), i32p, vp, vp, vp, vp]
     lib.dapq_evict_host.restype = C.c_int
     lib.dapq_recall.argtypes = [vp, vp, vp, i32p, i32p, C.c_int32, f32p, vp]
@@ -241,7 +243,7 @@ def dapq_evict(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, cu_ro
 
 def dapq_evict_layers(ctx, q_pre: Sequence[torch.Tensor], k: Sequence[torch.Tensor], v: Sequence[torch.Tensor], cu_rows,
                       prompt_len, k_keep, k_out: Sequence[torch.Tensor], v_out: Sequence[torch.Tensor],
-                      idx_out: Optional[Sequence[torch.Tensor]] = None, stream=None) -> None:
+                      idx_out: Optional[Sequence[torch.Tensor]] = None, stream=None, host: bool = False) -> None:
     """k_keep: one budget row [batch] for all layers, or one row per layer [n_layers][batch]."""
     n = len(k)
     views = (dapq_cache_view * n)()
@@ -256,8 +258,13 @@ def dapq_evict_layers(ctx, q_pre: Sequence[torch.Tensor], k: Sequence[torch.Tens
     stride = budgets.shape[1] if budgets.ndim == 2 else 0
     arr = lambda ts: (C.c_void_p * n)(*[t.data_ptr() for t in ts])
     idx_arr = arr(idx_out) if idx_out is not None else None
-    _check(ctx, load_library().dapq_evict_layers(ctx, n, arr(q_pre), views, kk_p, stride, arr(k_out), arr(v_out),
-                                                 idx_arr, _stream(stream)))
+    fn = load_library().dapq_evict_layers_host if host else load_library().dapq_evict_layers
+    _check(ctx, fn(ctx, n, arr(q_pre), views, kk_p, stride, arr(k_out), arr(v_out), idx_arr, _stream(stream)))
+
+
+def dapq_evict_layers_host(ctx, q_pre, k, v, cu_rows, prompt_len, k_keep, k_out, v_out, idx_out=None, stream=None) -> None:
+    """dapq_evict_layers on host tensors (pinned memory gives full copy speed); returns once the results are there."""
+    dapq_evict_layers(ctx, q_pre, k, v, cu_rows, prompt_len, k_keep, k_out, v_out, idx_out, stream, host=True)
 
 
 def dapq_evict_host(ctx, q_pre: torch.Tensor, k: torch.Tensor, v: torch.Tensor, cu_rows, prompt_len, k_keep,

@@ -29,9 +29,16 @@ struct dapq_ctx {
   float* scores = nullptr;       // [H_kv, max_total_rows]
   float* pooled = nullptr;       // [H_kv, max_total_rows] (pooling only)
   int32_t* idx = nullptr;        // [H_kv, max_total_rows]
-  // staging for dapq_evict_host (allocated on first use)
-  void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_ko = nullptr, *h_vo = nullptr;
-  int32_t* h_idx = nullptr;
+  // staging for the host-buffer entry points (allocated on first use): two sets, so that the copies of one
+  // layer run beside the kernels of the layer before
+  struct HostStage {
+    void *q = nullptr, *k = nullptr, *v = nullptr, *ko = nullptr, *vo = nullptr;
+    int32_t* idx = nullptr;
+    cudaEvent_t in_done = nullptr;    // the layer's inputs have arrived (recorded on the copy stream)
+    cudaEvent_t out_done = nullptr;   // the layer's results have left (recorded on the caller's stream)
+  } hs[2];
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t fork = nullptr;         // orders the copy stream behind what the caller's stream already holds
   LaunchLog log;
   char err[512] = "";
 };
@@ -310,10 +317,18 @@ void dapq_destroy(dapq_ctx* ctx) {
   if (!ctx) return;
   {
     DeviceGuard guard(ctx->device);
-    void* bufs[] = {ctx->inv_freq, ctx->status, ctx->q_rot, ctx->part, ctx->lse2, ctx->scores, ctx->pooled,
-                    ctx->idx, ctx->h_q, ctx->h_k, ctx->h_v, ctx->h_ko, ctx->h_vo, ctx->h_idx};
+    void* bufs[] = {ctx->inv_freq, ctx->status, ctx->q_rot, ctx->part, ctx->lse2, ctx->scores, ctx->pooled, ctx->idx};
     for (void* p : bufs)
       if (p) cudaFree(p);
+    for (auto& st : ctx->hs) {
+      void* sb[] = {st.q, st.k, st.v, st.ko, st.vo, st.idx};
+      for (void* p : sb)
+        if (p) cudaFree(p);
+      if (st.in_done) cudaEventDestroy(st.in_done);
+      if (st.out_done) cudaEventDestroy(st.out_done);
+    }
+    if (ctx->fork) cudaEventDestroy(ctx->fork);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   }
   delete static_cast<dapq::ProfImpl*>(ctx->log.impl);
   delete ctx;
@@ -518,87 +533,138 @@ dapq_status dapq_evict_layers(dapq_ctx* ctx, int32_t n_layers, const void* const
   return DAPQ_OK;
 }
 
-dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
-                            const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
-                            int32_t* idx_out_host, void* stream) {
+namespace {
+
+// First use of a staging set: its buffers (V only when some caller's V cannot be read in place) and events.
+dapq_status ensure_stage(dapq_ctx* ctx, int set, bool need_v) {
+  const dapq_shape& sh = ctx->shape;
+  dapq_ctx::HostStage& hs = ctx->hs[set];
+  const size_t row_bytes = (size_t)kHeadDim * ctx->elem_bytes;
+  const size_t cache_bytes = (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * row_bytes;
+  if (!ctx->copy_stream) {
+    DAPQ_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    DAPQ_CUDA(ctx, cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming));
+  }
+  if (!hs.k) {
+    DAPQ_CUDA(ctx, cudaMalloc(&hs.q, (size_t)sh.max_batch * sh.n_q_heads * sh.n_pseudo * row_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&hs.k, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&hs.ko, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&hs.vo, cache_bytes));
+    DAPQ_CUDA(ctx, cudaMalloc(&hs.idx, (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * sizeof(int32_t)));
+    DAPQ_CUDA(ctx, cudaEventCreateWithFlags(&hs.in_done, cudaEventDisableTiming));
+    DAPQ_CUDA(ctx, cudaEventCreateWithFlags(&hs.out_done, cudaEventDisableTiming));
+  }
+  if (need_v && !hs.v) DAPQ_CUDA(ctx, cudaMalloc(&hs.v, cache_bytes));
+  return DAPQ_OK;
+}
+
+// Device address of the caller's V if the compaction kernel can read it in place (page-locked, addressable
+// by the device, 16-byte geometry), else NULL.
+const void* mapped_v(dapq_ctx* ctx, const CacheDev& hv) {
+  cudaPointerAttributes pa;
+  const int per16 = 16 / ctx->elem_bytes;
+  if (hv.v_row_stride % per16 || hv.v_head_stride % per16) return nullptr;
+  if (cudaPointerGetAttributes(&pa, hv.v) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer &&
+      aligned16(pa.devicePointer))
+    return pa.devicePointer;
+  cudaGetLastError();
+  return nullptr;
+}
+
+}  // namespace
+
+dapq_status dapq_evict_layers_host(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre_host,
+                                   const dapq_cache_view* caches_host, const int32_t* k_keep_host,
+                                   int64_t k_keep_layer_stride, void* const* k_out_host, void* const* v_out_host,
+                                   int32_t* const* idx_out_host, void* stream) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
-  if (!q_pre_host || !k_keep_host || !k_out_host || !v_out_host)
-    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_host: NULL argument");
-  CacheDev hv;
-  dapq_status st = check_view(ctx, cache_host, true, true, &hv);
-  if (st != DAPQ_OK) return st;
-  SeqTable t;
-  st = build_table(ctx, cache_host->batch, cache_host->cu_rows_host, cache_host->prompt_len_host, nullptr,
-                   k_keep_host, nullptr, &t);
-  if (st != DAPQ_OK) return st;
+  if (n_layers < 0 || k_keep_layer_stride < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers_host: negative count or stride");
+  if (n_layers > 0 && (!q_pre_host || !caches_host || !k_keep_host || !k_out_host || !v_out_host))
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers_host: NULL argument");
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)stream;
   const dapq_shape& sh = ctx->shape;
   const size_t eb = (size_t)ctx->elem_bytes, row_bytes = (size_t)kHeadDim * eb;
-  if (!ctx->h_k) {
-    const size_t cache_bytes = (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * row_bytes;
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_q, (size_t)sh.max_batch * sh.n_q_heads * sh.n_pseudo * row_bytes));
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_k, cache_bytes));
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_v, cache_bytes));
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_ko, cache_bytes));
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_vo, cache_bytes));
-    DAPQ_CUDA(ctx, cudaMalloc(&ctx->h_idx, (size_t)sh.n_kv_heads * (size_t)sh.max_total_rows * sizeof(int32_t)));
+  bool forked = false;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    const int32_t* keep = k_keep_host + (int64_t)l * k_keep_layer_stride;
+    if (!q_pre_host[l] || !k_out_host[l] || !v_out_host[l]) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers_host: NULL layer pointer");
+    CacheDev hv;
+    dapq_status st = check_view(ctx, &caches_host[l], true, true, &hv);
+    if (st != DAPQ_OK) return st;
+    SeqTable t;
+    st = build_table(ctx, caches_host[l].batch, caches_host[l].cu_rows_host, caches_host[l].prompt_len_host, nullptr, keep,
+                     nullptr, &t);
+    if (st != DAPQ_OK) return st;
+    const void* v_in_place = mapped_v(ctx, hv);
+    const int set = l & 1;
+    st = ensure_stage(ctx, set, v_in_place == nullptr);
+    if (st != DAPQ_OK) return st;
+    dapq_ctx::HostStage& hs = ctx->hs[set];
+    cudaStream_t cs = ctx->copy_stream;
+    if (!forked) {                                       // the copies start behind the work already in `stream`
+      DAPQ_CUDA(ctx, cudaEventRecord(ctx->fork, s));
+      DAPQ_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->fork, 0));
+      forked = true;
+    }
+    if (l >= 2) DAPQ_CUDA(ctx, cudaStreamWaitEvent(cs, hs.out_done, 0));   // the set's last user is done with it
+    // ---- inputs: q and the used row range [cu_rows[0], cu_rows[B]) of every head of K, packed from row 0
+    const int64_t row0 = t.cu_rows[0], n_rows = t.cu_rows[t.batch] - row0;
+    DAPQ_CUDA(ctx, cudaMemcpyAsync(hs.q, q_pre_host[l], (size_t)t.batch * sh.n_q_heads * sh.n_pseudo * row_bytes,
+                                   cudaMemcpyHostToDevice, cs));
+    for (int h = 0; h < sh.n_kv_heads; ++h) {
+      const char* ks = (const char*)hv.k + ((size_t)h * hv.k_head_stride + (size_t)row0 * hv.k_row_stride) * eb;
+      DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)hs.k + (size_t)h * n_rows * row_bytes, row_bytes, ks,
+                                       (size_t)hv.k_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, cs));
+      if (v_in_place) continue;
+      const char* vs = (const char*)hv.v + ((size_t)h * hv.v_head_stride + (size_t)row0 * hv.v_row_stride) * eb;
+      DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)hs.v + (size_t)h * n_rows * row_bytes, row_bytes, vs,
+                                       (size_t)hv.v_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, cs));
+    }
+    DAPQ_CUDA(ctx, cudaEventRecord(hs.in_done, cs));
+    // ---- the layer itself, on the caller's stream
+    int32_t cu_local[kMaxBatch + 1];
+    for (int b = 0; b <= t.batch; ++b) cu_local[b] = (int32_t)(t.cu_rows[b] - row0);
+    dapq_cache_view dv;
+    memset(&dv, 0, sizeof(dv));
+    dv.k = hs.k;
+    dv.k_head_stride = n_rows * kHeadDim;
+    dv.k_row_stride = kHeadDim;
+    if (v_in_place) {
+      dv.v = (const char*)v_in_place + (size_t)row0 * hv.v_row_stride * eb;   // row 0 of the view = row cu_rows[0] of the caller's
+      dv.v_head_stride = hv.v_head_stride;
+      dv.v_row_stride = hv.v_row_stride;
+    } else {
+      dv.v = hs.v;
+      dv.v_head_stride = n_rows * kHeadDim;
+      dv.v_row_stride = kHeadDim;
+    }
+    dv.cu_rows_host = cu_local;
+    dv.prompt_len_host = caches_host[l].prompt_len_host;
+    dv.batch = t.batch;
+    DAPQ_CUDA(ctx, cudaStreamWaitEvent(s, hs.in_done, 0));
+    st = dapq_evict(ctx, hs.q, &dv, keep, hs.ko, hs.vo, hs.idx, nullptr, stream);
+    if (st != DAPQ_OK) return st;
+    // ---- results
+    const size_t kt = (size_t)t.cu_keep[t.batch];
+    DAPQ_CUDA(ctx, cudaMemcpyAsync(k_out_host[l], hs.ko, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
+    DAPQ_CUDA(ctx, cudaMemcpyAsync(v_out_host[l], hs.vo, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
+    if (idx_out_host && idx_out_host[l])
+      DAPQ_CUDA(ctx, cudaMemcpyAsync(idx_out_host[l], hs.idx, (size_t)sh.n_kv_heads * kt * sizeof(int32_t),
+                                     cudaMemcpyDeviceToHost, s));
+    DAPQ_CUDA(ctx, cudaEventRecord(hs.out_done, s));
   }
-  // Only the kept rows of V are needed.  If the caller's V is page-locked host memory that the device can
-  // address, the compaction kernel gathers those rows straight from it; otherwise V is staged like K.
-  const void* v_mapped = nullptr;
-  {
-    cudaPointerAttributes pa;
-    const int per16 = 16 / ctx->elem_bytes;                        // (the kernel reads 16-byte pieces)
-    const bool vector_ok = hv.v_row_stride % per16 == 0 && hv.v_head_stride % per16 == 0;
-    if (vector_ok && cudaPointerGetAttributes(&pa, hv.v) == cudaSuccess && pa.type == cudaMemoryTypeHost &&
-        pa.devicePointer && aligned16(pa.devicePointer))
-      v_mapped = pa.devicePointer;
-    else
-      cudaGetLastError();
-  }
-  // device copy of the used row range [cu_rows[0], cu_rows[B]) of every head, packed from row 0
-  const int64_t row0 = t.cu_rows[0], n_rows = t.cu_rows[t.batch] - row0;
-  DAPQ_CUDA(ctx, cudaMemcpyAsync(ctx->h_q, q_pre_host, (size_t)t.batch * sh.n_q_heads * sh.n_pseudo * row_bytes,
-                                 cudaMemcpyHostToDevice, s));
-  for (int h = 0; h < sh.n_kv_heads; ++h) {
-    const char* ks = (const char*)hv.k + ((size_t)h * hv.k_head_stride + (size_t)row0 * hv.k_row_stride) * eb;
-    DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_k + (size_t)h * n_rows * row_bytes, row_bytes, ks,
-                                     (size_t)hv.k_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
-    if (v_mapped) continue;
-    const char* vs = (const char*)hv.v + ((size_t)h * hv.v_head_stride + (size_t)row0 * hv.v_row_stride) * eb;
-    DAPQ_CUDA(ctx, cudaMemcpy2DAsync((char*)ctx->h_v + (size_t)h * n_rows * row_bytes, row_bytes, vs,
-                                     (size_t)hv.v_row_stride * eb, row_bytes, (size_t)n_rows, cudaMemcpyHostToDevice, s));
-  }
-  int32_t cu_local[kMaxBatch + 1];
-  for (int b = 0; b <= t.batch; ++b) cu_local[b] = (int32_t)(t.cu_rows[b] - row0);
-  dapq_cache_view dv;
-  memset(&dv, 0, sizeof(dv));
-  dv.k = ctx->h_k;
-  dv.k_head_stride = n_rows * kHeadDim;
-  dv.k_row_stride = kHeadDim;
-  if (v_mapped) {
-    dv.v = (const char*)v_mapped + (size_t)row0 * hv.v_row_stride * eb;     // row 0 of the view = row cu_rows[0] of the caller's
-    dv.v_head_stride = hv.v_head_stride;
-    dv.v_row_stride = hv.v_row_stride;
-  } else {
-    dv.v = ctx->h_v;
-    dv.v_head_stride = n_rows * kHeadDim;
-    dv.v_row_stride = kHeadDim;
-  }
-  dv.cu_rows_host = cu_local;
-  dv.prompt_len_host = cache_host->prompt_len_host;
-  dv.batch = t.batch;
-  st = dapq_evict(ctx, ctx->h_q, &dv, k_keep_host, ctx->h_ko, ctx->h_vo, ctx->h_idx, nullptr, stream);
-  if (st != DAPQ_OK) return st;
-  const size_t kt = (size_t)t.cu_keep[t.batch];
-  DAPQ_CUDA(ctx, cudaMemcpyAsync(k_out_host, ctx->h_ko, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
-  DAPQ_CUDA(ctx, cudaMemcpyAsync(v_out_host, ctx->h_vo, (size_t)sh.n_kv_heads * kt * row_bytes, cudaMemcpyDeviceToHost, s));
-  if (idx_out_host)
-    DAPQ_CUDA(ctx, cudaMemcpyAsync(idx_out_host, ctx->h_idx, (size_t)sh.n_kv_heads * kt * sizeof(int32_t),
-                                   cudaMemcpyDeviceToHost, s));
   DAPQ_CUDA(ctx, cudaStreamSynchronize(s));
   return DAPQ_OK;
+}
+
+dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
+                            const int32_t* k_keep_host, void* k_out_host, void* v_out_host,
+                            int32_t* idx_out_host, void* stream) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (!q_pre_host || !cache_host || !k_keep_host || !k_out_host || !v_out_host)
+    return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_host: NULL argument");
+  return dapq_evict_layers_host(ctx, 1, &q_pre_host, cache_host, k_keep_host, 0, &k_out_host, &v_out_host, &idx_out_host, stream);
 }
 
 }  // extern "C"

@@ -59,4 +59,5 @@ def test_null_context_is_an_error_not_a_crash(lib):
     assert cdll.dapq_poll_status(None, None) == lib.DAPQ_ERR_INVALID_ARG
     assert cdll.dapq_launch_count(None) == 0
     assert cdll.dapq_evict_layers(None, 0, None, None, None, 0, None, None, None, None) == lib.DAPQ_ERR_INVALID_ARG
+    assert cdll.dapq_evict_layers_host(None, 0, None, None, None, 0, None, None, None, None) == lib.DAPQ_ERR_INVALID_ARG
     cdll.dapq_destroy(None)

@@ -287,6 +287,26 @@ def test_evict_host_matches_device_call(dq, pinned):
     dq.dapq_destroy(ctx)
 
 
+def test_evict_layers_host_pipelines_five_layers(dq):
+    """The multi-layer host call (two staging sets, copies of one layer beside the kernels of the layer
+    before) equals a device call per layer, with per-layer budgets; layers 2..4 reuse the staging sets."""
+    lens, budgets = (900, 333), [(90, 33), (45, 10), (200, 60), (9, 3), (120, 50)]
+    ws, datas = _layer_cases(5, lens, budgets, n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
+    ctx = _ctx(dq, ws[0])
+    pin = lambda t: t.contiguous().pin_memory()
+    q, k, v = ([pin(d[x]) for d in datas] for x in ("q_pre", "k", "v"))
+    ko = [torch.empty((w.n_kv_heads, int(w.cu_keep[-1]), 128), dtype=torch.bfloat16).pin_memory() for w in ws]
+    vo = [torch.empty_like(t).pin_memory() for t in ko]
+    idx = [torch.empty((w.n_kv_heads, int(w.cu_keep[-1])), dtype=torch.int32).pin_memory() for w in ws]
+    dq.dapq_evict_layers_host(ctx, q, k, v, ws[0].cu_rows, ws[0].prompt_lens, budgets, ko, vo, idx)
+    dq.dapq_poll_status(ctx)
+    for l, (w, data) in enumerate(zip(ws, datas)):
+        one = _gpu_evict(dq, w, data, ctx)
+        np.testing.assert_array_equal(idx[l].numpy(), one["idx"])
+        assert torch.equal(ko[l], one["k_out"]) and torch.equal(vo[l], one["v_out"]), f"layer {l}"
+    dq.dapq_destroy(ctx)
+
+
 def test_argument_errors_launch_nothing(dq):
     w = _small(lens=(100,), keep=(10,), n_needles=0)
     data = gi.draw_layer(w, 0, "cuda")
