@@ -348,6 +348,8 @@ dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream) {
   if (word) DAPQ_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof(int)));
   if (word & kStatusTimeout) return fail(ctx, DAPQ_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its results are undefined");
   if (word & kStatusBadIndex) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_compact_kv skipped indices outside [0, L_b)");
+  if (word & kStatusSmemAlign)
+    return fail(ctx, DAPQ_ERR_UNSUPPORTED, "the score kernels found their shared memory off a 1024-byte boundary and did nothing");
   return DAPQ_OK;
 }
 

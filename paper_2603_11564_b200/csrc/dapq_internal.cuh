@@ -49,7 +49,7 @@ struct Dims {
 };
 
 // Device status word bits (set by kernels, read by dapq_poll_status).
-enum : int { kStatusTimeout = 1, kStatusBadIndex = 2 };
+enum : int { kStatusTimeout = 1, kStatusBadIndex = 2, kStatusSmemAlign = 4 };
 
 // Output formats of the rotation kernel.
 enum : int { kRopeOutBf16 = DAPQ_BF16, kRopeOutF32 = DAPQ_F32, kRopeOutSplitBf16 = 2 };

@@ -5,9 +5,10 @@
 // A job is one [128 keys x 256 queries] accumulator (two fit; four of 128 columns in the compact
 // geometry).  All four epilogue groups work
 // on every job, a quarter of the query columns each (sixteen epilogue warps, four per scheduler,
-// hide the latency of the tensor-memory loads and of the hand-offs); groups 1-3 hand their
-// partial sums to group 0 through consumed columns of the same accumulator, and group 0's thread
-// (lane = key) stores the key's score: one coalesced fp32 per lane.  Before the first job the
+// hide the latency of the tensor-memory loads and of the hand-offs) and gives the accumulator back
+// as soon as its columns are in registers; groups 1-3 hand their partial sums to group 0 through
+// shared memory, and group 0's thread (lane = key) stores the key's score: one coalesced fp32 per
+// lane.  Before the first job the
 // epilogue threads merge the per-chunk partials of sweep 1 into the base-2 log-sum-exp of the
 // resident query rows.
 #pragma once
@@ -21,9 +22,12 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                     const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
                     const __grid_constant__ ChunkTable ct1, const UmmaArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {                                          // (uniform over the CTA: nothing has been set up yet)
+    if (threadIdx.x == 0) atomicOr(a.status, kStatusSmemAlign);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   using G = Geo<kCompact>;
   constexpr int kStages2 = G::kStages2, kAcc = G::kAcc2, kAccCols = G::kAccCols2;
@@ -34,6 +38,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   const Bars bars{sbase + Smem::bars};
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
   float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
+  float* exch = reinterpret_cast<float*>(smem + Smem::exch);    // [3][128] partial sums on their way to group 0
   const uint32_t tmem_base = cta_prologue(smem, sbase, bars, kStages2, kAcc);
 
   if (warp == 0) {
@@ -85,7 +90,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2e;
     const float2 c2 = make_float2(c, c);
-    int job = 0;
+    int job = 0;                                                // jobs of this CTA so far
     bool ok = true;
     // (an aborting group still walks every query group: the other groups wait for it at the barriers)
     for (int qg = 0; qg < a.n_qgroups; ++qg) {
@@ -142,12 +147,20 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tc_fence_after();
         const uint32_t taddr = lane_addr + buf * kAccCols;
         float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+        // the accumulator goes back to the MMA issuer as soon as this warp's last piece is in registers
+        auto release = [&] {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+        };
+        if (np == 0) release();
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           if (k < np) {
             uint32_t v[32];
             tmem_ld32(taddr + (p0 + k) * 32, v);
             tmem_ld_wait_for(v);
+            if (k == np - 1) release();
             const int ch = p0 + k;
             const int valid = rows_g - ch * 32;                 // >= 32 except in the last piece
             if (valid >= 32) {
@@ -170,32 +183,21 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           }
         }
         float sum = (acc.x + acc.y) + (acc1.x + acc1.y);
+        // Groups 1-3 hand their partial sums to group 0 through one slot of shared memory: the slot is
+        // written once group 0 has read the job before (part_empty) and read once all three have
+        // written (part_full).
         if (eg > 0) {
-          // hand the partial sum over in the first column this group has consumed (nothing to hand over
-          // if it had no columns), then release the accumulator
-          if (np > 0) {
-            tmem_st1(taddr + p0 * 32, __float_as_uint(sum));
-            tmem_st_wait();
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) { mbar_arrive(bars.half_done(buf)); mbar_arrive(bars.acc_empty(buf)); }
-        } else {
-          ok = __all_sync(0xffffffffu, mbar_wait(bars.half_done(buf), (job / kAcc) & 1, abort_flag, a.status));
+          if (job > 0) ok = __all_sync(0xffffffffu, mbar_wait(bars.part_empty(), (job - 1) & 1, abort_flag, a.status));
           if (!ok) break;
-          tc_fence_after();
-          // the three partial sums: loads issued together, one wait (a group without columns left nothing)
-          uint32_t part[kEpiGroups - 1] = {0u, 0u, 0u};
-#pragma unroll
-          for (int g = 1; g < kEpiGroups; ++g) {
-            const int gp0 = (g * nch) / kEpiGroups, gnp = ((g + 1) * nch) / kEpiGroups - gp0;
-            if (gnp > 0) tmem_ld1_issue(taddr + gp0 * 32, part[g - 1]);
-          }
-          tmem_ld_wait3(part[0], part[1], part[2]);
-          sum += (__uint_as_float(part[0]) + __uint_as_float(part[1])) + __uint_as_float(part[2]);
-          tc_fence_before();
+          exch[(eg - 1) * 128 + r] = sum;
           __syncwarp();
-          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+          if (lane == 0) mbar_arrive(bars.part_full());         // (release: the stores above are visible to the waiter)
+        } else {
+          ok = __all_sync(0xffffffffu, mbar_wait(bars.part_full(), job & 1, abort_flag, a.status));
+          if (!ok) break;
+          sum += (exch[r] + exch[128 + r]) + exch[256 + r];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.part_empty());
           const int j = (w.t0 + ti) * kTile2 + r;               // sequence-local key position
           if (j < L) {
             float* out = a.scores + (int64_t)kvh * a.score_stride + t.cu_prompt[b] + j;

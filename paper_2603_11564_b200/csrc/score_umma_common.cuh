@@ -40,9 +40,10 @@ constexpr int kMaxStages = 3, kMaxAcc = 4;
 // (sweep 2) and two words.
 struct Smem {
   static constexpr int bars = 224 * 1024;
-  // barriers (20 x 8 B): k_full[3], k_empty[3], acc_full[4], acc_empty[4], q_full, q_empty, half_done[4]
-  static constexpr int lse = bars + 20 * 8;          // [256] floats
-  static constexpr int tmem_ptr = lse + 256 * 4;
+  // barriers (18 x 8 B): k_full[3], k_empty[3], acc_full[4], acc_empty[4], q_full, q_empty, part_full, part_empty
+  static constexpr int lse = bars + 18 * 8;          // [256] floats
+  static constexpr int exch = lse + 256 * 4;         // [3][128] floats: the partial sums of epilogue groups 1-3 (sweep 2)
+  static constexpr int tmem_ptr = exch + 3 * 128 * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -50,7 +51,9 @@ static_assert(Geo<false>::k + Geo<false>::kStages1 * kStageBytes1 <= Smem::bars 
               Geo<false>::k + Geo<false>::kStages2 * kStageBytes2 <= Smem::bars && Geo<true>::k + Geo<true>::kStages2 * kStageBytes2 <= Smem::bars,
               "K ring overruns the barriers");
 static_assert(Geo<true>::kStages1 <= kMaxStages && Geo<true>::kStages2 <= kMaxStages && Geo<true>::kAcc2 <= kMaxAcc, "barrier table too small");
-constexpr int kSmemBytes = Smem::total + 1024;   // slack for the manual 1024-byte alignment
+// The kernels declare their dynamic shared memory 1024-byte aligned (what the 128-byte swizzle of the
+// TMA / UMMA tiles needs) and check it: a CTA that finds it otherwise raises a status bit and returns.
+constexpr int kSmemBytes = Smem::total;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
 struct UmmaArgs {
@@ -98,7 +101,8 @@ struct Bars {
   __device__ __forceinline__ uint32_t acc_empty(int i) const { return base + 8u * (2 * kMaxStages + kMaxAcc + i); }
   __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc); }
   __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 1); }
-  __device__ __forceinline__ uint32_t half_done(int i) const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 2 + i); }
+  __device__ __forceinline__ uint32_t part_full() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 2); }
+  __device__ __forceinline__ uint32_t part_empty() const { return base + 8u * (2 * kMaxStages + 2 * kMaxAcc + 3); }
 };
 
 // Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync, then
@@ -111,8 +115,9 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
     for (int i = 0; i < n_acc; ++i) {
       mbar_init(bars.acc_full(i), 1);
       mbar_init(bars.acc_empty(i), 4 * kEpiGroups);        // every epilogue warp reads every accumulator
-      mbar_init(bars.half_done(i), 4 * (kEpiGroups - 1));  // the groups that hand their partial sums to group 0
     }
+    mbar_init(bars.part_full(), 4 * (kEpiGroups - 1));     // the groups that hand their partial sums to group 0
+    mbar_init(bars.part_empty(), 4);                       // group 0 has read them
     mbar_init(bars.q_full(), 1);
     mbar_init(bars.q_empty(), 1);
     *reinterpret_cast<volatile int*>(smem + Smem::abort_flag) = 0;
