@@ -51,14 +51,18 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
   }
 }
 
-// This group's 48 columns of one accumulator, in three 16-column pieces.
+// This group's 48 columns of one accumulator, in three 16-column pieces; `release` gives the accumulator
+// back once the last piece is in registers.
+template <class Release>
 __device__ __forceinline__ void row_stats_job(uint32_t taddr, int col0, bool masked, int lim, float c, float& m_raw,
-                                              float& z) {
+                                              float& z, Release release) {
+  constexpr int kPieces = kTile1 / kEpiGroups / 16;
 #pragma unroll
-  for (int ch = 0; ch < kTile1 / kEpiGroups / 16; ++ch) {
+  for (int ch = 0; ch < kPieces; ++ch) {
     uint32_t v[16];
     tmem_ld16(taddr + ch * 16, v);
     tmem_ld_wait_for16(v);
+    if (ch == kPieces - 1) release();
     if (masked) row_stats_piece<true>(v, col0 + ch * 16, lim, c, m_raw, z);
     else row_stats_piece<false>(v, col0 + ch * 16, lim, c, m_raw, z);
   }
@@ -164,11 +168,13 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           tc_fence_after();
           const uint32_t taddr = lane_addr + buf * kTile1 + col0;
           // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
-          if (m == 0) row_stats_job(taddr, col0, masked, L + i_q0 - tile_base, c, m_raw0, z0);
-          else row_stats_job(taddr, col0, masked, L + i_q1 - tile_base, c, m_raw1, z1);
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+          auto release = [&] {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+          };
+          if (m == 0) row_stats_job(taddr, col0, masked, L + i_q0 - tile_base, c, m_raw0, z0, release);
+          else row_stats_job(taddr, col0, masked, L + i_q1 - tile_base, c, m_raw1, z1, release);
         }
       }
       // partials: slot eg of this thread's rows
