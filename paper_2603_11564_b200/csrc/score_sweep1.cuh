@@ -7,10 +7,10 @@
 // accumulator each, so the MMAs of one block run while the other block's accumulator is read
 // (a group of one block alternates between the two accumulators from tile to tile).
 // All four epilogue groups work on every job, 48 key columns each: thread (group g, row r) keeps
-// the statistics of query row r over the columns of its group, which become slot g of the
-// row's per-chunk partials.  Sixteen epilogue warps (four per scheduler) hide the latency of
-// the tensor-memory loads and of the hand-offs, so each reads its columns in plain 16-column
-// pieces.
+// the statistics of query row r over the columns of its group; at the end of a chunk the four
+// groups fold their statistics together through shared memory into the row's per-chunk partial.
+// Sixteen epilogue warps (four per scheduler) hide the latency of the tensor-memory loads and of
+// the hand-offs, so each reads its columns in plain 16-column pieces.
 #pragma once
 #include "score_umma_common.cuh"
 
@@ -49,6 +49,13 @@ __device__ __forceinline__ void row_stats_piece(const uint32_t* v, int col0, int
     }
     z += (acc0.x + acc0.y) + (acc1.x + acc1.y);
   }
+}
+
+// (max, sum of exp2) of two disjoint sets of logits -> of their union.
+__device__ __forceinline__ float2 merge_stats(float2 a, float2 b) {
+  const float m = fmaxf(a.x, b.x);
+  if (m == -CUDART_INF_F) return make_float2(m, 0.f);
+  return make_float2(m, a.y * exp2f(a.x - m) + b.y * exp2f(b.x - m));
 }
 
 // This group's 48 columns of one accumulator, in three 16-column pieces; `release` gives the accumulator
@@ -149,8 +156,10 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const float c = a.scale_log2e;
     const int col0 = eg * (kTile1 / kEpiGroups);
     uint32_t use0 = 0u, use1 = 0u;                              // jobs taken from each accumulator
+    float2* stat = reinterpret_cast<float2*>(smem + Smem::lse);  // [256] (max, sum) of the rows on their way through the groups
     bool ok = true;
-    for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
+    // (an aborting warp still walks every query group: the others wait for it at the barriers)
+    for (int qg = 0; qg < a.n_qgroups; ++qg) {
       const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
       const int mb = (rows_g + 127) / 128;
       // running max (raw dot product) and sum of this thread's row of block 0 / block 1
@@ -167,20 +176,40 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           if (buf) ++use1; else ++use0;
           tc_fence_after();
           const uint32_t taddr = lane_addr + buf * kTile1 + col0;
-          // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
           auto release = [&] {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bars.acc_empty(buf));
           };
+          // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
           if (m == 0) row_stats_job(taddr, col0, masked, L + i_q0 - tile_base, c, m_raw0, z0, release);
           else row_stats_job(taddr, col0, masked, L + i_q1 - tile_base, c, m_raw1, z1, release);
         }
       }
-      // partials: slot eg of this thread's rows
-      float2* pbase = a.part + (((int64_t)chunk * a.n_kv_heads + kvh) * kEpiGroups + eg) * a.rows_pad + qg * G::kRows;
-      if (qg * G::kRows + r < a.rows_total) pbase[r] = make_float2(m_raw0 * c, z0);
-      if (mb == 2 && qg * G::kRows + 128 + r < a.rows_total) pbase[128 + r] = make_float2(m_raw1 * c, z1);
+      // The four groups hold the statistics of the same rows over different key columns: group 3 puts its
+      // pair into shared memory, groups 2 and 1 fold theirs in, group 0 folds last and stores the chunk's
+      // partials (a fixed order, so the result does not depend on timing).
+      float2 s0 = make_float2(m_raw0 * c, z0), s1 = make_float2(m_raw1 * c, z1);
+      if (qg > 0) epilogue_sync();                              // group 0 has read the round before
+#pragma unroll
+      for (int g = kEpiGroups - 1; g >= 0; --g) {
+        if (eg == g) {
+          if (g < kEpiGroups - 1) {
+            s0 = merge_stats(s0, stat[r]);
+            s1 = merge_stats(s1, stat[128 + r]);
+          }
+          if (g > 0) {
+            stat[r] = s0;
+            stat[128 + r] = s1;
+          }
+        }
+        if (g > 0) epilogue_sync();
+      }
+      if (eg == 0) {
+        float2* pbase = a.part + ((int64_t)chunk * a.n_kv_heads + kvh) * a.rows_pad + qg * G::kRows;
+        if (qg * G::kRows + r < a.rows_total) pbase[r] = s0;
+        if (mb == 2 && qg * G::kRows + 128 + r < a.rows_total) pbase[128 + r] = s1;
+      }
     }
   }
   cta_epilogue(tmem_base);

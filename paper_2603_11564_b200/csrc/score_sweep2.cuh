@@ -95,46 +95,55 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     // (an aborting group still walks every query group: the other groups wait for it at the barriers)
     for (int qg = 0; qg < a.n_qgroups; ++qg) {
       const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
-      // ---- base-2 log-sum-exp of the group's rows: thread (eg, r) merges the per-chunk
-      // partials of row eg*128 + r in a fixed order, or converts the caller's value
+      // ---- base-2 log-sum-exp of the group's rows.  Two threads per row: thread (eg, r) merges the per-chunk
+      // partials of row (eg & 1) * 128 + r over the chunks of parity eg >> 1, all of its loads in flight at
+      // once; the odd half then crosses through shared memory and the even half finishes (fixed order).
       if (qg > 0) epilogue_sync();                              // the previous group's values are no longer read
-      if (eg * 128 < G::kRows) {
-        const int row = eg * 128 + r, grow = qg * G::kRows + row;
-        float l2 = 0.f;
-        if (grow < a.rows_total) {
-          if (a.lse_in) {
-            l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
-          } else {
-            const int rows_pad = a.rows_pad;
-            const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * kEpiGroups * rows_pad + grow;
-            const int64_t step = (int64_t)a.n_kv_heads * kEpiGroups * rows_pad;
-            const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
-            // one pass, sixteen independent loads in flight; (max, sum) merged in chunk order
-            float mx = -CUDART_INF_F, z = 0.f;
-            for (int c0 = 0; c0 < nc; c0 += 4) {
-              float2 q[16];
+      {
+        const int row = (eg & 1) * 128 + r, grow = qg * G::kRows + row;
+        const bool live = row < G::kRows && grow < a.rows_total;
+        float mx = -CUDART_INF_F, z = 0.f;
+        if (live && !a.lse_in) {
+          const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * a.rows_pad + grow;
+          const int64_t step = (int64_t)a.n_kv_heads * a.rows_pad;
+          const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
+          for (int c0 = eg >> 1; c0 < nc; c0 += 32) {
+            float2 q[16];
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const bool in = c0 + u < nc;
+            for (int u = 0; u < 16; ++u)
+              q[u] = c0 + 2 * u < nc ? __ldg(p + (c0 + 2 * u) * step) : make_float2(-CUDART_INF_F, 0.f);
+            float m16 = q[0].x;
 #pragma unroll
-                for (int g = 0; g < kEpiGroups; ++g)
-                  q[kEpiGroups * u + g] = in ? __ldg(p + (c0 + u) * step + g * rows_pad) : make_float2(-CUDART_INF_F, 0.f);
-              }
-              float m8 = q[0].x;
-#pragma unroll
-              for (int u = 1; u < 16; ++u) m8 = fmaxf(m8, q[u].x);
-              if (m8 > mx) {
-                z *= exp2f(mx - m8);                        // exp2f(-inf) = 0 on the first chunk
-                mx = m8;
-              }
+            for (int u = 1; u < 16; ++u) m16 = fmaxf(m16, q[u].x);
+            if (m16 > mx) {
+              z *= exp2f(mx - m16);                             // exp2f(-inf) = 0 on the first round
+              mx = m16;
+            }
+            if (mx > -CUDART_INF_F) {
 #pragma unroll
               for (int u = 0; u < 16; ++u) z += q[u].y * exp2f(q[u].x - mx);
             }
-            l2 = mx + log2f(z);
           }
-          if (a.lse_out && chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
         }
-        lse_s[row] = -l2;                                         // negated: the epilogue adds it
+        if (eg >= 2) {                                          // (lse_s holds the odd half's sums until the even half has read them)
+          exch[row] = mx;
+          lse_s[row] = z;
+        }
+        epilogue_sync();
+        if (eg < 2) {
+          float l2 = 0.f;
+          if (live) {
+            if (a.lse_in) {
+              l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
+            } else {
+              const float mo = exch[row], zo = lse_s[row];
+              const float m = fmaxf(mx, mo);
+              l2 = m + log2f(z * exp2f(mx - m) + zo * exp2f(mo - m));
+            }
+            if (a.lse_out && chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
+          }
+          lse_s[row] = -l2;                                       // negated: the epilogue adds it
+        }
       }
       epilogue_sync();
       // 32-column pieces of a job: group g takes pieces [g nch / 4, (g + 1) nch / 4)

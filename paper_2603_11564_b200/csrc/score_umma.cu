@@ -110,7 +110,7 @@ bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int n_kv_head
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo) {
   const int rows_total = n_q_heads / n_kv_heads * n_pseudo;
   const int rows_pad = (rows_total + 255) / 256 * 256;          // (the compact geometry pads to 128: never more)
-  return (int64_t)(max_batch + kUmmaMaxChunks) * n_kv_heads * kEpiGroups * rows_pad;
+  return (int64_t)(max_batch + kUmmaMaxChunks) * n_kv_heads * rows_pad;
 }
 
 bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheDev& cv, const SeqTable& t,

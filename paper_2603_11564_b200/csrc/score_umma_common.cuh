@@ -42,7 +42,8 @@ struct Smem {
   static constexpr int bars = 224 * 1024;
   // barriers (18 x 8 B): k_full[3], k_empty[3], acc_full[4], acc_empty[4], q_full, q_empty, part_full, part_empty
   static constexpr int lse = bars + 18 * 8;          // [256] floats
-  static constexpr int exch = lse + 256 * 4;         // [3][128] floats: the partial sums of epilogue groups 1-3 (sweep 2)
+  static constexpr int exch = lse + 256 * 4;         // [3][128] floats: the partial sums of epilogue groups 1-3 (sweep 2);
+                                                     // lse + exch together: [256] float2 row statistics (sweep 1)
   static constexpr int tmem_ptr = exch + 3 * 128 * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
@@ -64,7 +65,7 @@ struct UmmaArgs {
   int32_t has_lo;            // the query operand carries a low-order bf16 part
   int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
   float scale_log2e;
-  float2* part;              // [n_chunks1, H_kv, 4, rows_pad] (running max, sum) in base 2, one slot per group
+  float2* part;              // [n_chunks1, H_kv, rows_pad] (running max, sum) of every query row over a chunk's keys, base 2
   const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
   float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
   float* scores;
