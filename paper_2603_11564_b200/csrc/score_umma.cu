@@ -24,9 +24,11 @@
 // 77 cycles whatever its size, so MMAs are made wide (N = 192 / 256: 105 / 139 cycles for
 // 128 x N x 16) and their descriptors cost one add each; a commit -> wait -> release -> issue
 // hand-off of an accumulator takes about 700 cycles, so a job is a whole [128 x 192 / 256]
-// block of 16 MMAs and all epilogue groups split the columns of every job, which shortens the
-// time an accumulator is held; four epilogue warps per scheduler hide the ~370-cycle latency
-// of a tensor-memory load and the hand-off waits behind each other's exponentials.
+// block of 16 MMAs, all epilogue groups split the columns of every job, and a warp gives the
+// accumulator back the moment its last columns are in registers (what it still owes, the
+// exponentials and the exchange of partial sums, needs no tensor memory).  With that, sweep 2
+// runs at the pace of its MMAs; sweep 1 at the pace of its epilogue (maximum, rescaling and
+// exponentials of 16 columns take a warp ~600 cycles with all sixteen at work).
 //
 // CTA = (chunk of K tiles, KV head); 18 warps: warp 0 issues the TMA loads (query group, K
 // ring), warp 1 issues the MMAs and owns tensor memory, warps 2-17 are four epilogue groups
