@@ -15,7 +15,9 @@
  *   3. dapq_topk_select    M_retain = TopK_j S(j)                       (Section 4.2, Eq. 5)
  *   4. dapq_compact_kv     keep the K/V rows in M_retain, drop the rest and every
  *                          synthetic token (Section 4.2, last paragraph; Figure 1).
- *   5. dapq_evict          1-4 for one layer's cache on one stream (dapq_evict_layers: every layer).
+ *   5. dapq_evict          1-4 for one layer's cache on one stream (dapq_evict_layers: every layer;
+ *                          dapq_evict_host, dapq_evict_layers_host: the same on host buffers).
+ *   Also: dapq_recall (Section 3.3, Eq. 1-3), optional pooling of the scores before step 3.
  *
  * Conventions
  *   - One process drives one GPU.  All kernels are asynchronous on the caller's
@@ -23,7 +25,8 @@
  *   - "device" pointers are caller-owned device memory that must stay valid until
  *     the stream work finishes; "host" pointers are read before the call returns.
  *   - The library allocates device memory only inside dapq_create (workspace sized
- *     from dapq_shape) and, on first use, inside dapq_evict_host (staging buffers).
+ *     from dapq_shape) and, on first use, inside dapq_evict_host / dapq_evict_layers_host
+ *     (staging buffers, a copy stream, events).
  *   - Argument errors are returned synchronously and launch nothing.  A bounded
  *     device-side wait that gives up sets a status word that dapq_poll_status reads.
  *   - Outputs must not alias inputs.
