@@ -3,7 +3,10 @@
 //
 //   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
 // A job is one [128 keys x 256 queries] accumulator (two fit; four of 128 columns in the compact
-// geometry).  All four epilogue groups work
+// geometry).  In the compact geometry with a hi + lo query operand (kWide) the 128 hi rows and the
+// 128 lo rows sit side by side as the 256 columns of ONE MMA per k-step: the K tile is read from
+// shared memory once instead of twice (MMAs of N = 128 with both operands in shared memory are
+// bound by its bandwidth), and the epilogue adds the two halves before the exponential.  All four epilogue groups work
 // on every job, a quarter of the query columns each (sixteen epilogue warps, four per scheduler,
 // hide the latency of the tensor-memory loads and of the hand-offs) and gives the accumulator back
 // as soon as its columns are in registers; groups 1-3 hand their partial sums to group 0 through
@@ -17,7 +20,7 @@
 namespace dapq {
 namespace umma {
 
-template <bool kCompact>
+template <bool kCompact, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                     const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
@@ -30,7 +33,8 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   using G = Geo<kCompact>;
-  constexpr int kStages2 = G::kStages2, kAcc = G::kAcc2, kAccCols = G::kAccCols2;
+  static_assert(kCompact || !kWide, "the side-by-side operand needs the compact geometry");
+  constexpr int kStages2 = G::kStages2, kAcc = kWide ? 2 : G::kAcc2, kAccCols = kTmemCols / kAcc;
   const int chunk = blockIdx.x, kvh = blockIdx.y;
   const Work w = cta_work(t, ct, a, kTile2, false);
   const int nt = w.nt, L = w.L, b = w.b;
@@ -43,7 +47,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 
   if (warp == 0) {
     if (lane == 0)
-      tma_producer<G, kTile2, kStages2, kStageBytes2, kHalfBytes2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
+      tma_producer<G, kTile2, kStages2, kStageBytes2, kHalfBytes2, kWide>(&tm_k, &tm_q, w, a, sbase, bars, kvh, abort_flag);
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
@@ -52,7 +56,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       const uint64_t qd_hi = umma_desc(sbase + G::q_hi), qd_lo = umma_desc(sbase + G::q_lo);
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
         const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
-        const uint32_t idesc = umma_idesc(128, (rows_g + 15) & ~15);   // only the query columns that exist
+        const uint32_t idesc = umma_idesc(128, kWide ? 256 : (rows_g + 15) & ~15);   // only the query columns that exist
         ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
         for (int ti = 0; ti < nt && ok; ++ti, ++job) {
           const int s = job % kStages2, buf = job % kAcc;
@@ -62,18 +66,28 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           tc_fence_after();
           const uint64_t kd = umma_desc(sbase + G::k + s * kStageBytes2);
           const uint32_t d = tmem_base + buf * kAccCols;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const int half = ks >> 2, kk = ks & 3;
-            umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * G::kHalfBytesQ + kk * 32),
-                    idesc, ks ? 1u : 0u);
-          }
-          if (a.has_lo) {
+          if (kWide) {
+            // hi and lo rows side by side: one MMA of N = 256 per k-step, columns 0-127 = K q_hi^T, 128-255 = K q_lo^T
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const int half = ks >> 2, kk = ks & 3;
-              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_lo, half * G::kHalfBytesQ + kk * 32),
-                      idesc, 1u);
+              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * 2 * G::kHalfBytesQ + kk * 32),
+                      idesc, ks ? 1u : 0u);
+            }
+          } else {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const int half = ks >> 2, kk = ks & 3;
+              umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_hi, half * G::kHalfBytesQ + kk * 32),
+                      idesc, ks ? 1u : 0u);
+            }
+            if (a.has_lo) {
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const int half = ks >> 2, kk = ks & 3;
+                umma_ss(d, desc_advance(kd, half * kHalfBytes2 + kk * 32), desc_advance(qd_lo, half * G::kHalfBytesQ + kk * 32),
+                        idesc, 1u);
+              }
             }
           }
           tc_commit(bars.acc_full(buf));
@@ -146,8 +160,10 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
       }
       epilogue_sync();
-      // 32-column pieces of a job: group g takes pieces [g nch / 4, (g + 1) nch / 4)
-      const int nch = (rows_g + 31) >> 5;
+      // Pieces of a job (32 query columns; 16 with the side-by-side operand, whose two halves are added
+      // first): group g takes pieces [g nch / 4, (g + 1) nch / 4), at most two
+      constexpr int kPiece = kWide ? 16 : 32;
+      const int nch = (rows_g + kPiece - 1) / kPiece;
       const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
       for (int ti = 0; ti < nt && ok; ++ti, ++job) {
         const int buf = job % kAcc;
@@ -166,28 +182,55 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           if (k < np) {
-            uint32_t v[32];
-            tmem_ld32(taddr + (p0 + k) * 32, v);
-            tmem_ld_wait_for(v);
-            if (k == np - 1) release();
             const int ch = p0 + k;
-            const int valid = rows_g - ch * 32;                 // >= 32 except in the last piece
-            if (valid >= 32) {
-              // pairs of columns on the packed fp32 pipe: x = s * c - lse, then 2^x by MUFU or polynomial
+            const int valid = rows_g - ch * kPiece;             // >= kPiece except in the last piece
+            if (kWide) {
+              uint32_t vh[16], vl[16];
+              tmem_ld16(taddr + ch * 16, vh);                   // K q_hi^T
+              tmem_ld16(taddr + 128 + ch * 16, vl);             // K q_lo^T
+              tmem_ld_wait_for16(vh);
+              tmem_ld_wait_for16(vl);
+              if (k == np - 1) release();
+              if (valid >= 16) {
 #pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
-                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2,
-                                             make_float2(l4.x, l4.y));
-                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2,
-                                             make_float2(l4.z, l4.w));
-                acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
-                acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
+                for (int e = 0; e < 16; e += 4) {
+                  const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 16 + e);
+                  const float2 s0 = __fadd2_rn(make_float2(__uint_as_float(vh[e]), __uint_as_float(vh[e + 1])),
+                                               make_float2(__uint_as_float(vl[e]), __uint_as_float(vl[e + 1])));
+                  const float2 s1 = __fadd2_rn(make_float2(__uint_as_float(vh[e + 2]), __uint_as_float(vh[e + 3])),
+                                               make_float2(__uint_as_float(vl[e + 2]), __uint_as_float(vl[e + 3])));
+                  const float2 x0 = __ffma2_rn(s0, c2, make_float2(l4.x, l4.y));
+                  const float2 x1 = __ffma2_rn(s1, c2, make_float2(l4.z, l4.w));
+                  acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
+                  acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                  if (e < valid) acc.x += ex2(fmaf(__uint_as_float(vh[e]) + __uint_as_float(vl[e]), c, lse_s[ch * 16 + e]));
               }
             } else {
+              uint32_t v[32];
+              tmem_ld32(taddr + ch * 32, v);
+              tmem_ld_wait_for(v);
+              if (k == np - 1) release();
+              if (valid >= 32) {
+                // pairs of columns on the packed fp32 pipe: x = s * c - lse, then 2^x by MUFU or polynomial
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[e]), c, lse_s[ch * 32 + e]));
+                for (int e = 0; e < 32; e += 4) {
+                  const float4 l4 = *reinterpret_cast<const float4*>(lse_s + ch * 32 + e);
+                  const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2,
+                                               make_float2(l4.x, l4.y));
+                  const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2,
+                                               make_float2(l4.z, l4.w));
+                  acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
+                  acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[e]), c, lse_s[ch * 32 + e]));
+              }
             }
           }
         }

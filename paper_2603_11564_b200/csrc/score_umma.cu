@@ -173,8 +173,9 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
     log->end(s);
     return cudaSuccess;
   };
-  const cudaError_t e = compact ? run(score_sweep1_kernel<true>, score_sweep2_kernel<true>)
-                                : run(score_sweep1_kernel<false>, score_sweep2_kernel<false>);
+  const cudaError_t e = !compact      ? run(score_sweep1_kernel<false>, score_sweep2_kernel<false, false>)
+                        : plan.has_lo ? run(score_sweep1_kernel<true>, score_sweep2_kernel<true, true>)
+                                      : run(score_sweep1_kernel<true>, score_sweep2_kernel<true, false>);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }

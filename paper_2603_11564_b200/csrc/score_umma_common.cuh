@@ -147,7 +147,9 @@ __device__ __forceinline__ void cta_epilogue(uint32_t tmem_base) {
 
 // TMA producer loop shared by both sweeps: per query group the query blocks (hi, lo), then the
 // CTA's K tiles through the ring.  kTile / kStages / kHalf are the sweep's tile geometry.
-template <class G, int kTile, int kStages, int kStage, int kHalf>
+// kSideBySide (compact geometry only): per 64-channel half, the 128 hi rows are followed directly by the
+// 128 lo rows, so that one MMA of N = 256 reads both.
+template <class G, int kTile, int kStages, int kStage, int kHalf, bool kSideBySide = false>
 __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w,
                                              const UmmaArgs& a, uint32_t sbase, const Bars& bars, int kvh,
                                              volatile int* abort_flag) {
@@ -176,8 +178,9 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     for (int part = 0; part < parts; ++part)
       for (int half = 0; half < 2; ++half)
         for (int m = 0; m < mb; ++m)
-          tma_load_2d(sbase + (part ? G::q_lo : G::q_hi) + half * G::kHalfBytesQ + m * 128 * 128, tm_q, bars.q_full(),
-                      half * 64, part * a.lo_row_offset + w.qrow_base + qg * G::kRows + m * 128);
+          tma_load_2d(sbase + (kSideBySide ? half * 2 * G::kHalfBytesQ + part * G::kHalfBytesQ
+                                           : (part ? G::q_lo : G::q_hi) + half * G::kHalfBytesQ + m * 128 * 128),
+                      tm_q, bars.q_full(), half * 64, part * a.lo_row_offset + w.qrow_base + qg * G::kRows + m * 128);
     for (int ti = (qg == 0 ? n_first : 0); ti < w.nt; ++ti) {
       const int s = li % kStages;
       if (li >= kStages) ok = mbar_wait(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status);
