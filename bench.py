@@ -45,11 +45,11 @@ FALLBACK_BF16_TFLOPS = 1590.0
 NCU_TRAFFIC_BYTES = {
     # profiles/evict_kernels_llama3_8b_32k.md (a 2-layer run of the same command; traffic per launch does not
     # depend on the number of layers)
-    ("sweep1", "llama3_8b_32k"): 68333568 + 1029632,
-    ("sweep2", "llama3_8b_32k"): 68497664 + 1016576,
+    ("sweep1", "llama3_8b_32k"): 68334336 + 904192,
+    ("sweep2", "llama3_8b_32k"): 68497152 + 988928,
     # profiles/evict_kernels_batched_serving.md
-    ("sweep1", "batched_serving"): 315074048 + 4145408,
-    ("sweep2", "batched_serving"): 313692416 + 6921472,
+    ("sweep1", "batched_serving"): 315074048 + 3527936,
+    ("sweep2", "batched_serving"): 313671936 + 6923776,
 }
 
 
