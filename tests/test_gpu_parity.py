@@ -287,13 +287,14 @@ def test_evict_host_matches_device_call(dq, pinned):
     dq.dapq_destroy(ctx)
 
 
-def test_evict_layers_host_pipelines_five_layers(dq):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_evict_layers_host_pipelines_five_layers(dq, pinned):
     """The multi-layer host call (two staging sets, copies of one layer beside the kernels of the layer
     before) equals a device call per layer, with per-layer budgets; layers 2..4 reuse the staging sets."""
     lens, budgets = (900, 333), [(90, 33), (45, 10), (200, 60), (9, 3), (120, 50)]
     ws, datas = _layer_cases(5, lens, budgets, n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0)
     ctx = _ctx(dq, ws[0])
-    pin = lambda t: t.contiguous().pin_memory()
+    pin = (lambda t: t.contiguous().pin_memory()) if pinned else (lambda t: t.contiguous().clone())   # pageable: V is staged too
     q, k, v = ([pin(d[x]) for d in datas] for x in ("q_pre", "k", "v"))
     ko = [torch.empty((w.n_kv_heads, int(w.cu_keep[-1]), 128), dtype=torch.bfloat16).pin_memory() for w in ws]
     vo = [torch.empty_like(t).pin_memory() for t in ko]
