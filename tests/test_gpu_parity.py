@@ -605,3 +605,13 @@ def test_evict_random_shapes(dq, dtype, hq, hkv, n, lens, keep):
                outlier_channels=2 if dtype == "bf16" else 0)
     data = gi.draw_layer(w, 0, "cpu")
     _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+
+
+def test_evict_largest_batch(dq):
+    """DAPQ_MAX_BATCH sequences in one call (1 to 300 tokens each, some keeping every row)."""
+    rng = np.random.default_rng(77)
+    lens = tuple(int(x) for x in rng.integers(1, 301, 128))
+    keep = tuple(int(min(L, max(1, rng.integers(1, 2 * L)))) for L in lens)
+    w = _small(lens=lens, keep=keep, n_q_heads=8, n_kv_heads=2, n_pseudo=16, n_needles=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
