@@ -280,7 +280,7 @@ class Env:
 
 
 def measure(env: Env, w: gi.Workload, n_layers: int, steps: int, warmup: int, repeats: int, min_seconds: float,
-            e2e_steps: int):
+            e2e_steps: int, flags: int = 0):
     """Build the workload's caches in HBM, time `steps` steps of dapq_evict_layers (CUDA events, max over
     ranks), then the same steps with every kernel bracketed by events.  Returns the measurement as a dict."""
     dq, dev, peaks = env.dq, env.dev, env.peaks
@@ -288,7 +288,7 @@ def measure(env: Env, w: gi.Workload, n_layers: int, steps: int, warmup: int, re
     dt = w.torch_dtype()
     KT = int(w.cu_keep[-1])
     ctx = dq.dapq_create(w.n_q_heads, w.n_kv_heads, w.n_pseudo, w.batch, w.total_rows,
-                         dq.DAPQ_BF16 if w.dtype == "bf16" else dq.DAPQ_F32, w.rope_base, device=env.local)
+                         dq.DAPQ_BF16 if w.dtype == "bf16" else dq.DAPQ_F32, w.rope_base, device=env.local, flags=flags)
 
     # ---- synthetic caches, resident in HBM; structure planted with the library's own rotation
     layers = []
@@ -479,7 +479,7 @@ def run_ours(args, w: gi.Workload):
     n_layers = args.layers or w.n_layers
     warmup = max(args.warmup, 3)
     head = measure(env, w, n_layers, args.steps, warmup, args.repeats, args.min_seconds,
-                   0 if args.no_e2e else max(1, args.e2e_steps))
+                   0 if args.no_e2e else max(1, args.e2e_steps), args.flags)
 
     # ---- the other configurations, briefly (caches of one freed before the next is built)
     sweep = None
@@ -489,7 +489,7 @@ def run_ours(args, w: gi.Workload):
             if name == w.name:
                 continue
             ws = gi.workload(name)
-            m = measure(env, ws, ws.n_layers, 5, 3, 1, args.sweep_seconds, 0)
+            m = measure(env, ws, ws.n_layers, 5, 3, 1, args.sweep_seconds, 0, args.flags)
             r = m["roofline"]
             sweep[name] = {
                 "us_per_layer": round(m["us_per_layer"], 2), "value": m["value"], "steps": m["steps"],
@@ -512,7 +512,7 @@ def run_ours(args, w: gi.Workload):
             "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": head["steps"],
             "warmup": warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": workload_config(w, n_layers, world),
+            "config": workload_config(w, n_layers, world, **({"flags": args.flags} if args.flags else {})),
             "us_per_layer": head["us_per_layer"], "timed_region_s": head["timed_region_s"],
             "repeats_ms_per_step": head["repeats_ms_per_step"], "us_per_layer_x_mhz": head["us_per_layer_x_mhz"],
             "host_us_per_layer": head["host_us_per_layer"],
@@ -538,6 +538,7 @@ def main():
                          "not given, since a shorter region runs at burst clocks; 0 with --steps)")
     ap.add_argument("--sweep-seconds", type=float, default=1.0, help="length of each other configuration's timed region")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--flags", type=int, default=0, help="dapq_shape.flags of the contexts (0: the library's defaults)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="measure the chosen configuration only")

@@ -83,8 +83,24 @@ typedef enum { DAPQ_POOL_NONE = 0, DAPQ_POOL_MAX = 1, DAPQ_POOL_AVG = 2 } dapq_p
  * (fp32 arithmetic on unrounded rotated queries) even where the tensor-core path applies.
  * DAPQ_FLAG_ROPE_INTERLEAVED: the rotation pairs channel 2c with 2c + 1 instead of c with
  * c + d/2 (Section 4.1 only says "RoPE"; the rotate-half pairing of the paper's Llama and Qwen
- * models is the default; the cache's keys must have been rotated with the same pairing). */
-typedef enum { DAPQ_FLAG_CUDA_CORE_SCORER = 1, DAPQ_FLAG_ROPE_INTERLEAVED = 2 } dapq_flags;
+ * models is the default; the cache's keys must have been rotated with the same pairing).
+ *
+ * Precision of the rotated queries on the tensor-core path of dapq_evict (the paper states no
+ * precision; Eq. 4 is evaluated with fp32 accumulation whatever the choice):
+ *   default                 queries rounded to fp16 (11 significant bits), fp16 x fp16 MMAs, the bf16
+ *                           keys converted to fp16 on the fly: exact for key magnitudes 2^-14 .. 65504,
+ *                           larger keys saturate at 65504;
+ *   DAPQ_FLAG_Q_BF16        queries rounded to bf16 (8 significant bits), bf16 x bf16 MMAs: any key
+ *                           magnitude, the coarsest scores (caches with outlier channels can leave
+ *                           the 2e-3 per-token band);
+ *   DAPQ_FLAG_Q_LO_SWEEP1,  queries as a bf16 pair hi + lo (16 significant bits); the named sweep(s)
+ *   DAPQ_FLAG_Q_LO_SWEEP2   (1 = row normalisers, 2 = column sums) add the lo part with a second MMA
+ *                           pass: any key magnitude, the finest scores, twice the tensor work in
+ *                           those sweeps.  Either flag implies bf16 queries. */
+typedef enum {
+  DAPQ_FLAG_CUDA_CORE_SCORER = 1, DAPQ_FLAG_ROPE_INTERLEAVED = 2, DAPQ_FLAG_Q_BF16 = 4, DAPQ_FLAG_Q_LO_SWEEP1 = 8,
+  DAPQ_FLAG_Q_LO_SWEEP2 = 16
+} dapq_flags;
 
 typedef struct dapq_ctx dapq_ctx;
 
@@ -134,6 +150,14 @@ DAPQ_API dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream);
 /* Number of kernels this context has launched so far (for benchmarks' accounting). */
 DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
 
+/* Diagnostics (the paper has no counterpart): the bound, in SM clock cycles, on every device-side
+ * wait of the tensor-core score kernels launched from now on; 0 restores the default (about one
+ * second).  A wait that outlasts the bound makes its CTA raise the timeout status, see its copies and
+ * MMAs in flight complete and return; dapq_poll_status then reports DAPQ_ERR_TIMEOUT and the
+ * call's results are undefined.  A bound of a few cycles makes every kernel give up at once, which is
+ * how the give-up path is tested. */
+DAPQ_API dapq_status dapq_set_wait_limit(dapq_ctx* ctx, int64_t cycles);
+
 /* Per-kernel timing for benchmarks (the paper has no counterpart).  While enabled, every
  * kernel launch is bracketed by CUDA events on its stream; dapq_profile(ctx, 1) also clears
  * the totals.  dapq_profile_read synchronises `stream` and returns, per kernel kind, the
@@ -141,10 +165,22 @@ DAPQ_API int64_t dapq_launch_count(const dapq_ctx* ctx);
  * enabled.  ms_out / count_out: host [DAPQ_PROF_KINDS], in the order of dapq_prof_kind. */
 typedef enum {
   DAPQ_PROF_ROPE = 0, DAPQ_PROF_SWEEP1 = 1, DAPQ_PROF_LSE_MERGE = 2, DAPQ_PROF_SWEEP2 = 3,
-  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_POOL = 6, DAPQ_PROF_RECALL = 7, DAPQ_PROF_KINDS = 8
+  DAPQ_PROF_TOPK = 4, DAPQ_PROF_COMPACT = 5, DAPQ_PROF_POOL = 6, DAPQ_PROF_RECALL = 7, DAPQ_PROF_SLOT_SUM = 8,
+  DAPQ_PROF_KINDS = 9
 } dapq_prof_kind;
 DAPQ_API dapq_status dapq_profile(dapq_ctx* ctx, int32_t enable);
 DAPQ_API dapq_status dapq_profile_read(dapq_ctx* ctx, void* stream, double* ms_out, int64_t* count_out);
+
+/* Frequency table of the Llama-3.1 long-context RoPE scaling, for dapq_shape.inv_freq_host (the
+ * paper's efficiency runs, Appendix B.6, use Llama-3.1-8B-Instruct, whose keys are rotated with these
+ * frequencies; Section 4.1 needs the pseudo queries rotated the same way).  Per channel pair c, with
+ * theta_c = rope_base^(-2c/d) and wavelength 2 pi / theta_c: wavelengths below original_context /
+ * high_freq_factor keep theta_c, those above original_context / low_freq_factor get theta_c / factor,
+ * the band between is interpolated linearly in original_context / wavelength.  Llama-3.1 uses
+ * rope_base 500000, factor 8, low 1, high 4, original_context 8192.
+ * inv_freq_out: host [DAPQ_HEAD_DIM / 2].  Host arithmetic only; touches no device. */
+DAPQ_API dapq_status dapq_rope_inv_freq_llama3(double rope_base, double factor, double low_freq_factor,
+                                      double high_freq_factor, int32_t original_context, double* inv_freq_out);
 
 /* Section 4.1: q_rot[b,h,i,:] = RoPE(q_pre[b,h,i,:], position pos_start[b] + i), rotate-half
  * pairing (channel c with c + d/2), angles formed in double precision.

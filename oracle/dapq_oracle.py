@@ -32,6 +32,31 @@ def rope_inv_freq(head_dim: int, rope_base: float) -> np.ndarray:
     return np.power(np.float64(rope_base), -2.0 * c / np.float64(head_dim))
 
 
+def rope_inv_freq_llama3(head_dim: int, rope_base: float, factor: float = 8.0,
+                         low_freq_factor: float = 1.0, high_freq_factor: float = 4.0,
+                         original_context: int = 8192) -> np.ndarray:
+    """Frequencies of the Llama-3.1 long-context RoPE scaling (the model of the paper's efficiency
+    runs, Appendix B.6, is Llama-3.1-8B-Instruct).  The published rule, per channel pair c with
+    theta_c = base^(-2c/d) and wavelength lambda_c = 2 pi / theta_c:
+      lambda_c < original_context / high_freq_factor   -> theta_c unchanged (fast channels)
+      lambda_c > original_context / low_freq_factor    -> theta_c / factor  (slow channels)
+      in between                                       -> ((1 - s) / factor + s) * theta_c  with
+          s = (original_context / lambda_c - low_freq_factor) / (high_freq_factor - low_freq_factor).
+    """
+    theta = rope_inv_freq(head_dim, rope_base)
+    out = np.empty_like(theta)
+    for c in range(theta.shape[0]):
+        wavelen = 2.0 * math.pi / theta[c]
+        if wavelen < original_context / high_freq_factor:
+            out[c] = theta[c]
+        elif wavelen > original_context / low_freq_factor:
+            out[c] = theta[c] / factor
+        else:
+            s_ = (original_context / wavelen - low_freq_factor) / (high_freq_factor - low_freq_factor)
+            out[c] = ((1.0 - s_) / factor + s_) * theta[c]
+    return out
+
+
 def rope_pseudo_q(q_pre: np.ndarray, pos_start: int, rope_base: float,
                   inv_freq: Optional[np.ndarray] = None, interleaved: bool = False) -> np.ndarray:
     """Rotate pseudo queries to positions pos_start + i (Section 4.1, position assignment).

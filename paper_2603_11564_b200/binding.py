@@ -23,11 +23,12 @@ DAPQ_BF16, DAPQ_F32 = 0, 1
 DAPQ_POOL_NONE, DAPQ_POOL_MAX, DAPQ_POOL_AVG = 0, 1, 2
 DAPQ_FLAG_CUDA_CORE_SCORER = 1
 DAPQ_FLAG_ROPE_INTERLEAVED = 2
+DAPQ_FLAG_Q_BF16, DAPQ_FLAG_Q_LO_SWEEP1, DAPQ_FLAG_Q_LO_SWEEP2 = 4, 8, 16
 _STATUS_NAMES = {0: "DAPQ_OK", 1: "DAPQ_ERR_INVALID_ARG", 2: "DAPQ_ERR_UNSUPPORTED",
                  3: "DAPQ_ERR_WORKSPACE", 4: "DAPQ_ERR_CUDA", 5: "DAPQ_ERR_TIMEOUT"}
 
 EXPORTS = ("dapq_create", "dapq_destroy", "dapq_last_error", "dapq_poll_status",
-           "dapq_launch_count", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
+           "dapq_launch_count", "dapq_set_wait_limit", "dapq_rope_inv_freq_llama3", "dapq_profile", "dapq_profile_read", "dapq_rope_pseudo_q", "dapq_score", "dapq_topk_select",
            "dapq_compact_kv", "dapq_evict", "dapq_evict_layers", "dapq_evict_host", "dapq_evict_layers_host", "dapq_score_static", "dapq_recall")
 
 
@@ -75,6 +76,10 @@ def load_library() -> C.CDLL:
     lib.dapq_poll_status.restype = C.c_int
     lib.dapq_launch_count.argtypes = [vp]
     lib.dapq_launch_count.restype = C.c_int64
+    lib.dapq_rope_inv_freq_llama3.argtypes = [C.c_double, C.c_double, C.c_double, C.c_double, C.c_int32, C.POINTER(C.c_double)]
+    lib.dapq_rope_inv_freq_llama3.restype = C.c_int
+    lib.dapq_set_wait_limit.argtypes = [vp, C.c_int64]
+    lib.dapq_set_wait_limit.restype = C.c_int
     lib.dapq_profile.argtypes = [vp, C.c_int32]
     lib.dapq_profile.restype = C.c_int
     lib.dapq_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -178,7 +183,21 @@ def dapq_launch_count(ctx) -> int:
     return int(load_library().dapq_launch_count(ctx))
 
 
-PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact", "pool", "recall")
+PROF_KINDS = ("rope", "sweep1", "lse_merge", "sweep2", "topk", "compact", "pool", "recall", "slot_sum")
+
+
+def dapq_rope_inv_freq_llama3(rope_base: float = 5.0e5, factor: float = 8.0, low_freq_factor: float = 1.0,
+                              high_freq_factor: float = 4.0, original_context: int = 8192):
+    """[64] float64 frequencies for dapq_create(inv_freq=...)."""
+    out = (C.c_double * 64)()
+    st = load_library().dapq_rope_inv_freq_llama3(rope_base, factor, low_freq_factor, high_freq_factor, original_context, out)
+    if st != DAPQ_OK:
+        raise DapqError(st, "dapq_rope_inv_freq_llama3: bad argument")
+    return [float(x) for x in out]
+
+
+def dapq_set_wait_limit(ctx, cycles: int) -> None:
+    _check(ctx, load_library().dapq_set_wait_limit(ctx, int(cycles)))
 
 
 def dapq_profile(ctx, enable: bool) -> None:

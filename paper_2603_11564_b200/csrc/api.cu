@@ -28,6 +28,8 @@ struct dapq_ctx {
   float* lse2 = nullptr;         // [max_batch, H_q, N]
   float* scores = nullptr;       // [H_kv, max_total_rows]
   float* pooled = nullptr;       // [H_kv, max_total_rows] (pooling only)
+  float* slots = nullptr;        // [query groups, H_kv, max_total_rows] (only when a KV head has more than 256 query rows)
+  long long wait_limit = 0;      // cycles a device-side wait may take (0: the default, about a second)
   int32_t* idx = nullptr;        // [H_kv, max_total_rows]
   // staging for the host-buffer entry points (allocated on first use): two sets, so that the copies of one
   // layer run beside the kernels of the layer before
@@ -207,9 +209,21 @@ dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& 
                            float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
   cudaError_t e = launch_score_umma(plan, t, ctx->dims, lse_in, ctx->part, scores, score_stride,
                                     lse_out, ctx->status, s, &ctx->log);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels (two-part bf16 queries)");
+  return DAPQ_OK;
+}
+
+dapq_status run_score_qg(dapq_ctx* ctx, const QgPlan& plan, const SeqTable& t, const float* lse_in,
+                         float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
+  cudaError_t e = launch_score_qg(plan, t, ctx->dims, lse_in, ctx->part, ctx->slots, scores, score_stride, lse_out,
+                                  ctx->status, ctx->wait_limit, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels");
   return DAPQ_OK;
 }
+
+// The older tensor-core kernels (a second MMA pass with the low-order bf16 part of the queries) serve
+// the contexts that ask for that part in either sweep.
+bool wants_lo(const dapq_ctx* ctx) { return (ctx->shape.flags & (DAPQ_FLAG_Q_LO_SWEEP1 | DAPQ_FLAG_Q_LO_SWEEP2)) != 0; }
 
 dapq_status run_score(dapq_ctx* ctx, int q_dtype, const void* q_rot, const CacheDev& cd, const SeqTable& t,
                       const float* lse_in, float* scores, int64_t score_stride, float* lse_out,
@@ -259,7 +273,9 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   if (sh->max_batch > kMaxBatch || sh->max_total_rows > 0x7fffffffLL)
     return bail(DAPQ_ERR_UNSUPPORTED, "max_batch > 128 or max_total_rows >= 2^31");
   if (sh->dtype != DAPQ_BF16 && sh->dtype != DAPQ_F32) return bail(DAPQ_ERR_INVALID_ARG, "unknown dtype");
-  if (sh->flags & ~(DAPQ_FLAG_CUDA_CORE_SCORER | DAPQ_FLAG_ROPE_INTERLEAVED)) return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
+  if (sh->flags & ~(DAPQ_FLAG_CUDA_CORE_SCORER | DAPQ_FLAG_ROPE_INTERLEAVED | DAPQ_FLAG_Q_BF16 | DAPQ_FLAG_Q_LO_SWEEP1 |
+                    DAPQ_FLAG_Q_LO_SWEEP2))
+    return bail(DAPQ_ERR_INVALID_ARG, "unknown flag");
   if (sh->pool_mode != DAPQ_POOL_NONE && sh->pool_mode != DAPQ_POOL_MAX && sh->pool_mode != DAPQ_POOL_AVG)
     return bail(DAPQ_ERR_INVALID_ARG, "unknown pool_mode");
   if (sh->pool_mode != DAPQ_POOL_NONE && (sh->pool_kernel < 3 || sh->pool_kernel > DAPQ_MAX_POOL_KERNEL || sh->pool_kernel % 2 == 0))
@@ -306,6 +322,8 @@ dapq_status dapq_create(dapq_ctx** out, const dapq_shape* sh, int device) {
   ok = ok && cudaMalloc(&ctx->idx, (size_t)sh->n_kv_heads * rows * sizeof(int32_t)) == cudaSuccess;
   if (sh->pool_mode != DAPQ_POOL_NONE)
     ok = ok && cudaMalloc(&ctx->pooled, (size_t)sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
+  if (sh->dtype == DAPQ_BF16 && qg_groups(ctx->dims) > 1)
+    ok = ok && cudaMalloc(&ctx->slots, (size_t)qg_groups(ctx->dims) * sh->n_kv_heads * rows * sizeof(float)) == cudaSuccess;
   ok = ok && cudaMemcpy(ctx->inv_freq, freq, sizeof(freq), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemset(ctx->status, 0, sizeof(int)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); return bail(DAPQ_ERR_CUDA, "workspace allocation failed"); }
@@ -317,7 +335,7 @@ void dapq_destroy(dapq_ctx* ctx) {
   if (!ctx) return;
   {
     DeviceGuard guard(ctx->device);
-    void* bufs[] = {ctx->inv_freq, ctx->status, ctx->q_rot, ctx->part, ctx->lse2, ctx->scores, ctx->pooled, ctx->idx};
+    void* bufs[] = {ctx->inv_freq, ctx->status, ctx->q_rot, ctx->part, ctx->lse2, ctx->scores, ctx->pooled, ctx->slots, ctx->idx};
     for (void* p : bufs)
       if (p) cudaFree(p);
     for (auto& st : ctx->hs) {
@@ -337,6 +355,34 @@ void dapq_destroy(dapq_ctx* ctx) {
 const char* dapq_last_error(const dapq_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
 
 int64_t dapq_launch_count(const dapq_ctx* ctx) { return ctx ? ctx->log.n_launch : 0; }
+
+dapq_status dapq_rope_inv_freq_llama3(double rope_base, double factor, double low_freq_factor, double high_freq_factor,
+                                      int32_t original_context, double* inv_freq_out) {
+  if (!inv_freq_out || !(rope_base > 0.0) || !(factor >= 1.0) || !(low_freq_factor > 0.0) ||
+      !(high_freq_factor > low_freq_factor) || original_context < 1)
+    return DAPQ_ERR_INVALID_ARG;
+  const double two_pi = 6.283185307179586476925286766559;
+  const double short_wave = original_context / high_freq_factor, long_wave = original_context / low_freq_factor;
+  for (int c = 0; c < kHeadDim / 2; ++c) {
+    const double f = pow(rope_base, -2.0 * c / (double)kHeadDim), wave = two_pi / f;
+    double g = f;
+    if (wave > long_wave) {
+      g = f / factor;
+    } else if (wave >= short_wave) {
+      const double smooth = (original_context / wave - low_freq_factor) / (high_freq_factor - low_freq_factor);
+      g = (1.0 - smooth) * f / factor + smooth * f;
+    }
+    inv_freq_out[c] = g;
+  }
+  return DAPQ_OK;
+}
+
+dapq_status dapq_set_wait_limit(dapq_ctx* ctx, int64_t cycles) {
+  if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  if (cycles < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_set_wait_limit: negative limit");
+  ctx->wait_limit = cycles;
+  return DAPQ_OK;
+}
 
 dapq_status dapq_poll_status(dapq_ctx* ctx, void* stream) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
@@ -412,9 +458,16 @@ dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* 
   if (st != DAPQ_OK) return st;
   DeviceGuard guard(ctx->device);
   if (wants_umma(ctx) && !syn_mass) {
-    UmmaPlan plan;
-    if (umma_plan(q_rot, 0, 0, cd, t, ctx->dims, ctx->n_sm, &plan))
-      return run_score_umma(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, (cudaStream_t)stream);
+    // the caller's bf16 queries are exact in bf16: one bf16 x bf16 MMA pass, no conversion of K
+    if (wants_lo(ctx)) {
+      UmmaPlan plan;
+      if (umma_plan(q_rot, 0, 0, cd, t, ctx->dims, ctx->n_sm, &plan))
+        return run_score_umma(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, (cudaStream_t)stream);
+    } else {
+      QgPlan plan;
+      if (qg_plan(q_rot, 0, cd, t, ctx->dims, ctx->n_sm, &plan))
+        return run_score_qg(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, (cudaStream_t)stream);
+    }
   }
   return run_score(ctx, ctx->shape.dtype, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
 }
@@ -488,10 +541,22 @@ dapq_status evict_impl(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   int32_t* idx = idx_out ? idx_out : ctx->idx;
   const int64_t score_stride = t.cu_prompt[t.batch], idx_stride = t.cu_keep[t.batch];
   UmmaPlan plan;
+  QgPlan qplan;
   const int64_t lo_rows = ctx->q_rows_max;
+  const int flags = ctx->shape.flags;
   cudaError_t e;
-  if (wants_umma(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {
-    // tensor-core scorer: rotated queries as a bf16 pair hi + lo (two MMAs per k-step)
+  if (wants_umma(ctx) && !wants_lo(ctx) && qg_plan(ctx->q_rot, (flags & DAPQ_FLAG_Q_BF16) ? 0 : 1, cd, t, ctx->dims, ctx->n_sm, &qplan)) {
+    // tensor-core scorer: rotated queries rounded to fp16, K tiles converted to fp16 on their way to the MMAs
+    // (DAPQ_FLAG_Q_BF16: queries rounded to bf16, no conversion)
+    e = launch_rope(ctx->shape.dtype, qplan.q_is_f16 ? kRopeOutF16 : kRopeOutBf16, 0, q_pre, ctx->q_rot, ctx->inv_freq, t,
+                    ctx->dims, after_own_compaction, s, &ctx->log);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
+    st = run_score_qg(ctx, qplan, t, nullptr, scores, score_stride, nullptr, s);
+  } else if (wants_umma(ctx) && wants_lo(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {
+    // older tensor-core scorer: rotated queries as a bf16 pair hi + lo, the lo part added by a second MMA
+    // pass in the sweeps that the flags name
+    plan.lo_sweep1 = (flags & DAPQ_FLAG_Q_LO_SWEEP1) ? 1 : 0;
+    plan.lo_sweep2 = (flags & DAPQ_FLAG_Q_LO_SWEEP2) ? 1 : 0;
     e = launch_rope(ctx->shape.dtype, kRopeOutSplitBf16, lo_rows * kHeadDim, q_pre, ctx->q_rot, ctx->inv_freq, t,
                     ctx->dims, after_own_compaction, s, &ctx->log);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");

@@ -52,7 +52,7 @@ struct Dims {
 enum : int { kStatusTimeout = 1, kStatusBadIndex = 2, kStatusSmemAlign = 4 };
 
 // Output formats of the rotation kernel.
-enum : int { kRopeOutBf16 = DAPQ_BF16, kRopeOutF32 = DAPQ_F32, kRopeOutSplitBf16 = 2 };
+enum : int { kRopeOutBf16 = DAPQ_BF16, kRopeOutF32 = DAPQ_F32, kRopeOutSplitBf16 = 2, kRopeOutF16 = 3 };
 
 __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
   // largest b in [0, n) with cu[b] <= x
@@ -66,7 +66,7 @@ __device__ __forceinline__ int find_segment(const int32_t* cu, int n, int x) {
 
 // Kernel kinds, for launch accounting and the optional per-kernel event timing.
 enum KernelKind : int { kKindRope = 0, kKindSweep1, kKindLseMerge, kKindSweep2, kKindTopk, kKindCompact, kKindPool,
-                        kKindRecall, kKindCount };
+                        kKindRecall, kKindSlotSum, kKindCount };
 
 // Counts launches and, while profiling is on, brackets every launch with CUDA events on
 // the launching stream (implemented in api.cu; events come from a host-side pool).
@@ -142,7 +142,8 @@ cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const Ca
 struct UmmaPlan {
   CUtensorMap tm_k1, tm_k2, tm_q;   // K for sweep 1 / sweep 2 (different boxes), the query operand
   ChunkTable ct1, ct2;              // work cut of sweep 1 (192-key tiles over L_b + N) / sweep 2 (128-key tiles over L_b)
-  int32_t has_lo;
+  int32_t has_lo;                   // the low-order parts exist in memory
+  int32_t lo_sweep1, lo_sweep2;     // ... and which sweep adds them (a second MMA pass)
   int64_t lo_row_offset;
 };
 bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheDev& cv, const SeqTable& t,
@@ -151,6 +152,28 @@ int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseu
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
                               float2* part, float* scores, int64_t score_stride, float* lse_out,
                               int* status, cudaStream_t s, LaunchLog* log);
+
+// Pieces shared by the two tensor-core scorers (defined in score_qg.cu): the TMA descriptor of a
+// 16-bit [.., rows, 128] tensor (boxes of 64 channels x box_rows rows, 128-byte swizzle), and the cut of
+// the sequences' keys into chunks of whole tiles with ctas_per_chunk CTAs working on every chunk.
+bool encode_tile_map(CUtensorMap* map, const void* base, bool f16, int rank, const uint64_t* dims,
+                     const uint64_t* strides_bytes, int box_rows);
+bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_chunk, int n_sm, ChunkTable* ct);
+
+// Tensor-core scorer with one query group per CTA (score_qg.cu).  q: [B*H_q*N, d], fp16 (the K tiles
+// are then converted to fp16 in shared memory) or bf16.  qg_plan returns false when the view cannot be
+// described to TMA.  With more than one query group per KV head the sweeps write one score slot per
+// group into `slots` ([n_qgroups, H_kv, score_stride]) and a last kernel sums them into `scores`.
+struct QgPlan {
+  CUtensorMap tm_k1, tm_k2, tm_q;
+  ChunkTable ct1, ct2;
+  int32_t n_qgroups, rows_g, n_stages1, n_stages2, q_is_f16;
+};
+int qg_groups(const Dims& dm);
+bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t, const Dims& dm, int n_sm, QgPlan* plan);
+cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in, float2* part,
+                            float* slots, float* scores, int64_t score_stride, float* lse_out, int* status,
+                            long long wait_limit, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log);

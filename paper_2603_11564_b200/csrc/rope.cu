@@ -8,6 +8,8 @@
 // would cost half of the scorer's error budget.  Each thread evaluates its own sincos (the
 // table is tiny: B*N*64 angles), so no thread waits on another and the launch is one short
 // wave of independent loads and stores.
+#include <cuda_fp16.h>
+
 #include "dapq_internal.cuh"
 
 namespace dapq {
@@ -20,10 +22,15 @@ template <> __device__ __forceinline__ double to_double<float>(float x) { return
 template <> __device__ __forceinline__ double to_double<__nv_bfloat16>(__nv_bfloat16 x) {
   return (double)__bfloat162float(x);
 }
+template <> __device__ __forceinline__ double to_double<__half>(__half x) { return (double)__half2float(x); }
 template <typename T> __device__ __forceinline__ T from_double(double x);
 template <> __device__ __forceinline__ float from_double<float>(double x) { return (float)x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(double x) {
   return __double2bfloat16(x);
+}
+// fp16 output (the query operand of the fp16 MMAs): values beyond the format's range saturate
+template <> __device__ __forceinline__ __half from_double<__half>(double x) {
+  return __double2half(fmin(fmax(x, -65504.0), 65504.0));
 }
 
 // kSplit: TO is bf16 and the rounding residual is stored as a second bf16 lo_offset elements on.
@@ -75,6 +82,9 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
                (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw, dm.rope_interleaved);
+  } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutF16) {
+    launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __half, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
+               (__half*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
                (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);

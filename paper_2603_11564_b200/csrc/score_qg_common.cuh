@@ -22,7 +22,7 @@ constexpr int kThreads2 = kThreads1 + 32;                               // sweep
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 4, kMaxAcc = 4;
 constexpr int kExchDepth = 4;                  // jobs whose partial sums can wait in shared memory (sweep 2)
-constexpr int kRingEnd = 224 * 1024;           // queries + K ring end here; the small state follows
+constexpr int kRingEnd = 216 * 1024;           // queries + K ring end here; the small state follows
 
 template <int kTile>
 struct TileGeo {
@@ -101,6 +101,17 @@ struct Bars {
   __device__ __forceinline__ uint32_t drain() const { return base + 8u * (3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 1); }
 };
 
+// Position in a ring of n slots walked once per tile or job: slot index and the parity of its phase.
+struct Ring {
+  int n, i = 0;
+  uint32_t phase = 0;
+  bool wrapped = false;
+  __device__ __forceinline__ explicit Ring(int n_) : n(n_) {}
+  __device__ __forceinline__ void next() {
+    if (++i == n) { i = 0; phase ^= 1u; wrapped = true; }
+  }
+};
+
 // What a role needs to wait on a barrier: the CTA's abort flag, the status word, the cycle limit.
 struct Waiter {
   volatile int* abort_flag;
@@ -170,7 +181,7 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
   int li = 0;                                               // K tiles issued so far
   bool ok = true;
   auto load_tile = [&](int ti) {
-    const int s = ti % S;
+    const int s = li % S;                                   // (li == ti; one division per tile in this single thread)
     mbar_expect_tx(bars.k_full(s), T::kStage);
     const int row = w.row_base + (w.t0 + ti) * kTile;
     tma_load_3d(ring + s * T::kStage, tm_k, bars.k_full(s), 0, row, kvh);
@@ -183,20 +194,19 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     for (int m = 0; m < w.mb; ++m)
       tma_load_2d(sbase + half * (q_bytes / 2) + m * 128 * 128, tm_q, bars.q_full(), half * 64,
                   w.qrow_base + w.qgrp * a.rows_g + m * 128);
+  Ring rs(S);
   for (int ti = 1; ti < w.nt && ok; ++ti) {
-    const int s = ti % S;
-    if (ti >= S) ok = wt.wait(bars.k_empty(s), ((ti / S) - 1) & 1);
+    rs.next();
+    if (rs.wrapped) ok = wt.wait(bars.k_empty(rs.i), rs.phase ^ 1u);
     if (ok) load_tile(ti);
   }
-  if (!ok || wt.aborting()) {
-    // aborting: nobody may be left to consume the copies in flight; see them land before the CTA returns
-    const Waiter drain{wt.abort_flag, wt.status, kWaitLimit};
-    for (int back = 1; back <= S && back <= li; ++back) {
-      const int l2 = li - back;
-      drain_wait(bars.k_full(l2 % S), (l2 / S) & 1, kWaitLimit);
-    }
-    drain_wait(bars.q_full(), 0, kWaitLimit);
+  // See every copy issued above land before this thread (and with it the CTA) returns: in a normal run
+  // they have all been consumed by now; in an aborting CTA nobody else may be left to wait for them.
+  for (int back = 1; back <= S && back <= li; ++back) {
+    const int l2 = li - back;
+    drain_wait(bars.k_full(l2 % S), (l2 / S) & 1, kWaitLimit);
   }
+  drain_wait(bars.q_full(), 0, kWaitLimit);
 }
 
 // ---- K tiles from bf16 to fp16, in place (kConvWarps warps).  bf16 -> fp16 keeps every value of
@@ -219,9 +229,10 @@ __device__ __forceinline__ void convert_tiles(const Work& w, const Args& a, uint
   static_assert(kShare % (16 * 32) == 0 && kPieces % 4 == 0, "tile does not split over the converting warps");
   const int lane = threadIdx.x & 31, S = a.n_stages;
   const uint32_t ring = sbase + (uint32_t)w.mb * 2u * 128u * 128u;
-  for (int ti = 0; ti < w.nt; ++ti) {
-    const int s = ti % S;
-    if (!__all_sync(0xffffffffu, wt.wait(bars.k_full(s), (ti / S) & 1))) break;
+  Ring rs(S);
+  for (int ti = 0; ti < w.nt; ++ti, rs.next()) {
+    const int s = rs.i;
+    if (!__all_sync(0xffffffffu, wt.wait(bars.k_full(s), rs.phase))) break;
     const uint32_t p0 = ring + s * T::kStage + cw * kShare + lane * 16;
 #pragma unroll
     for (int it = 0; it < kPieces; it += 4) {

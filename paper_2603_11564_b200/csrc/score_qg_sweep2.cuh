@@ -1,0 +1,238 @@
+// Sweep 2 of the tensor-core scorer (Section 4.2, Eq. 4): S(j) = sum_i exp(s_ij - lse_i),
+// summed over the N pseudo queries and the G query heads of the KV head's group.
+//
+//   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
+// CTA = (chunk of K tiles, query group, KV head): a KV head with more than 256 query rows is cut into
+// groups of equal size, each scored by a CTA of its own against the same K chunk (the CTAs of a chunk
+// are neighbours in the grid, run at the same time and find each other's K tiles in L2, so K crosses
+// DRAM once); the groups' scores go to separate slots that a small kernel sums in fixed order.
+// A job is one [128 keys x <= 256 queries] accumulator (two fit; four of 128 columns for small groups).
+// All four epilogue groups work on every job, a quarter of the query columns each, and give the
+// accumulator back as soon as their columns are in registers.  No epilogue warp waits for another one:
+// a warp posts its 32 partial sums into a ring of kExchDepth slots in shared memory and goes on to the
+// next job; one more warp sums the four groups' entries (fixed order) and stores the keys' scores, one
+// coalesced fp32 per lane.  Before the first job the epilogue threads merge the per-chunk partials of
+// sweep 1 into the base-2 log-sum-exp of the resident query rows.
+#pragma once
+#include "score_qg_common.cuh"
+
+namespace dapq {
+namespace qg {
+
+// 16 accumulator columns of one key row: sum of 2^(s c - lse) over the columns, as two packed pairs.
+// kFull: all 16 columns exist (no per-column test).
+template <bool kFull>
+__device__ __forceinline__ void colsum_piece(const uint32_t* v, const float* lse16, int valid, float c, float2& acc, float2& acc1) {
+  if (kFull) {
+    const float2 c2 = make_float2(c, c);
+#pragma unroll
+    for (int e = 0; e < 16; e += 4) {
+      const float4 l4 = *reinterpret_cast<const float4*>(lse16 + e);
+      const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2, make_float2(l4.x, l4.y));
+      const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2, make_float2(l4.z, l4.w));
+      acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
+      acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[e]), c, lse16[e]));
+  }
+}
+
+// This warp's pieces [p0, p0 + np) of one accumulator (np <= 4), two at a time; `release` gives the
+// accumulator back once the last piece is in registers.  kFull: every column of these pieces exists.
+template <bool kFull, class Release>
+__device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, int p0, int np, int rows, float c, Release release) {
+  float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+  if (np == 0) release();
+#pragma unroll
+  for (int k = 0; k < 4; k += 2) {
+    if (k < np) {
+      const int ch = p0 + k;
+      const int valid = rows - ch * 16;                         // >= 16 except in the last piece
+      if (k + 1 < np) {
+        uint32_t v[32];
+        tmem_ld16(taddr + ch * 16, v);
+        tmem_ld16(taddr + ch * 16 + 16, v + 16);
+        tmem_ld_wait_for(v);
+        if (k + 2 >= np) release();
+        colsum_piece<kFull>(v, lse_s + ch * 16, valid, c, acc, acc1);
+        colsum_piece<kFull>(v + 16, lse_s + ch * 16 + 16, valid - 16, c, acc, acc1);
+      } else {
+        uint32_t v[16];
+        tmem_ld16(taddr + ch * 16, v);
+        tmem_ld_wait_for16(v);
+        release();
+        colsum_piece<kFull>(v, lse_s + ch * 16, valid, c, acc, acc1);
+      }
+    }
+  }
+  return (acc.x + acc.y) + (acc1.x + acc1.y);
+}
+
+template <bool kConvert>
+__global__ void __launch_bounds__(kThreads2, 1)
+colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+              const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
+              const __grid_constant__ ChunkTable ct1, const Args a) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {                                          // (uniform over the CTA: nothing has been set up yet)
+    if (threadIdx.x == 0) atomicOr(a.status, kStatusSmemAlign);
+    return;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  using T = TileGeo<kTile2>;
+  const int kvh = blockIdx.y;
+  const Work w = cta_work(t, ct, a, kTile2, false);
+  const int nt = w.nt, L = w.L, b = w.b;
+  if (nt <= 0) return;
+  const Bars bars{sbase + Smem::bars};
+  const Waiter wt{reinterpret_cast<volatile int*>(smem + Smem::abort_flag), a.status, a.wait_limit};
+  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
+  float* aux = reinterpret_cast<float*>(smem + Smem::aux);      // [256] scratch of the lse merge
+  float* exch = reinterpret_cast<float*>(smem + Smem::exch);    // [kExchDepth][4][128] partial sums on their way to the summing warp
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars);
+  const int ncols = (w.rows + 15) & ~15;                        // UMMA N: only the query columns that exist
+  const int acc_cols = ncols > 128 ? 256 : 128, n_acc = kTmemCols / acc_cols;
+  const uint32_t q_half = (uint32_t)w.mb * 128u * 128u;         // bytes of one 64-channel half of the query group
+  const int S = a.n_stages;
+
+  if (warp == 0) {
+    if (lane == 0) tma_producer<kTile2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+  } else if (warp == 1) {
+    // ============================================================================= MMA issuer
+    if (lane == 0) {
+      bool ok = wt.wait(bars.q_full(), 0);
+      const uint32_t idesc = kConvert ? umma_idesc_f16(128, ncols) : umma_idesc(128, ncols);
+      const uint64_t qd = umma_desc(sbase);
+      const uint32_t ring = sbase + 2 * q_half;
+      Ring rs(S), ra(n_acc);
+      for (int ti = 0; ti < nt && ok; ++ti, rs.next(), ra.next()) {
+        const int s = rs.i, buf = ra.i;
+        ok = wt.wait(kConvert ? bars.k_conv(s) : bars.k_full(s), rs.phase);
+        if (ok && ra.wrapped) ok = wt.wait(bars.acc_empty(buf), ra.phase ^ 1u);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t kd = umma_desc(ring + s * T::kStage);
+        const uint32_t d = tmem_base + buf * acc_cols;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const int half = ks >> 2, kk = ks & 3;
+          umma_ss(d, desc_advance(kd, half * T::kHalf + kk * 32), desc_advance(qd, half * q_half + kk * 32), idesc, ks ? 1u : 0u);
+        }
+        tc_commit(bars.acc_full(buf));
+        tc_commit(bars.k_empty(s));                             // the K stage is free once these MMAs retire
+      }
+      mma_drain(bars);
+    }
+  } else if (warp < kFirstEpiWarp) {
+    if (kConvert) convert_tiles<kTile2>(w, a, sbase, bars, warp - 2, wt);
+  } else if (warp < kFirstEpiWarp + 4 * kEpiGroups) {
+    // ============================================================================== epilogue
+    const int eg = (warp - kFirstEpiWarp) >> 2;                 // epilogue group 0 .. 3
+    const int quad = warp & 3;                                  // TMEM lane quadrant of this warp
+    const int r = quad * 32 + lane;                             // accumulator row (key) of this thread
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const float c = a.scale_log2e;
+    // ---- base-2 log-sum-exp of the group's rows.  Two threads per row: thread (eg, r) merges the per-chunk
+    // partials of row (eg & 1) * 128 + r over the chunks of parity eg >> 1, all of its loads in flight at
+    // once; the odd half then crosses through shared memory and the even half finishes (fixed order).
+    {
+      const int row = (eg & 1) * 128 + r, grow = w.qgrp * a.rows_g + row;
+      const bool live = row < w.rows;
+      float mx = -CUDART_INF_F, z = 0.f;
+      if (live && !a.lse_in) {
+        const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * a.rows_pad + grow;
+        const int64_t step = (int64_t)a.n_kv_heads * a.rows_pad;
+        const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
+        for (int c0 = eg >> 1; c0 < nc; c0 += 32) {
+          float2 q[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u)
+            q[u] = c0 + 2 * u < nc ? __ldg(p + (c0 + 2 * u) * step) : make_float2(-CUDART_INF_F, 0.f);
+          float m16 = q[0].x;
+#pragma unroll
+          for (int u = 1; u < 16; ++u) m16 = fmaxf(m16, q[u].x);
+          if (m16 > mx) {
+            z *= exp2f(mx - m16);                               // exp2f(-inf) = 0 on the first round
+            mx = m16;
+          }
+          if (mx > -CUDART_INF_F) {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) z += q[u].y * exp2f(q[u].x - mx);
+          }
+        }
+      }
+      if (eg >= 2) {
+        aux[row] = mx;
+        lse_s[row] = z;                                         // (the odd half's sums, until the even half has read them)
+      }
+      epilogue_sync();
+      if (eg < 2) {
+        float l2 = 0.f;
+        if (live) {
+          if (a.lse_in) {
+            l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
+          } else {
+            const float mo = aux[row], zo = lse_s[row];
+            const float m = fmaxf(mx, mo);
+            l2 = m + log2f(z * exp2f(mx - m) + zo * exp2f(mo - m));
+          }
+          if (a.lse_out && w.chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
+        }
+        lse_s[row] = -l2;                                       // negated: the epilogue adds it
+      }
+      epilogue_sync();
+    }
+    // Pieces of a job (16 query columns): group g takes pieces [g nch / 4, (g + 1) nch / 4), at most four
+    const int nch = ncols >> 4;
+    const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
+    const bool full = (p0 + np) * 16 <= w.rows;                 // no column of this warp's pieces lies beyond the group
+    bool ok = true;
+    Ring ra(n_acc);
+    for (int ti = 0; ti < nt && ok; ++ti, ra.next()) {
+      const int buf = ra.i;
+      ok = __all_sync(0xffffffffu, wt.wait(bars.acc_full(buf), ra.phase));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = lane_addr + buf * acc_cols;
+      // the accumulator goes back to the MMA issuer as soon as this warp's last piece is in registers
+      auto release = [&] {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+      };
+      const float sum = full ? colsum_job<true>(taddr, lse_s, p0, np, w.rows, c, release)
+                             : colsum_job<false>(taddr, lse_s, p0, np, w.rows, c, release);
+      const int slot = ti % kExchDepth;
+      if (ti >= kExchDepth) ok = __all_sync(0xffffffffu, wt.wait(bars.part_empty(slot), ((ti / kExchDepth) - 1) & 1));
+      if (!ok) break;
+      exch[(slot * kEpiGroups + eg) * 128 + r] = sum;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars.part_full(slot));         // (release: the stores above are visible to the waiter)
+    }
+  } else {
+    // ====================================================================== sum of the four groups
+    float* out = a.scores + (int64_t)w.qgrp * a.slot_stride + (int64_t)kvh * a.score_stride + t.cu_prompt[b];
+    for (int ti = 0; ti < nt; ++ti) {
+      const int slot = ti % kExchDepth;
+      if (!__all_sync(0xffffffffu, wt.wait(bars.part_full(slot), (ti / kExchDepth) & 1))) break;
+      const float* e = exch + slot * kEpiGroups * 128;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int r = q * 32 + lane;
+        const float v = ((e[r] + e[128 + r]) + e[256 + r]) + e[384 + r];
+        const int j = (w.t0 + ti) * kTile2 + r;                 // sequence-local key position
+        if (j < L) out[j] = v;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars.part_empty(slot));
+    }
+  }
+  cta_epilogue(tmem_base);
+}
+
+}  // namespace qg
+}  // namespace dapq

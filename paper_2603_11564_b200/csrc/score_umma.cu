@@ -43,70 +43,6 @@ namespace {
 
 using namespace umma;
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// bf16 tensor [.., rows, 128] with boxes of 64 channels x box_rows rows, 128-byte swizzle.
-bool encode_bf16_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                     int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gdim[3], gstride[2];
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1}, estr[3] = {1, 1, 1};
-  for (int i = 0; i < rank; ++i) gdim[i] = dims[i];
-  for (int i = 0; i < rank - 1; ++i) gstride[i] = strides_bytes[i];
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Cut every sequence's keys (prompt, plus the synthetic rows if asked) into chunks of whole tiles.
-bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int n_kv_heads, int n_sm, ChunkTable* ct) {
-  int max_tiles = 0;
-  for (int b = 0; b < t.batch; ++b) {
-    const int tiles = (t.prompt_len[b] + extra_keys + tile_keys - 1) / tile_keys;
-    max_tiles = tiles > max_tiles ? tiles : max_tiles;
-  }
-  // cost of a candidate = waves of CTAs x (tiles per CTA + fixed per-CTA work, in tile units)
-  int best_c = 0;
-  double best_cost = 0.0;
-  for (int c = 1; c <= max_tiles; ++c) {
-    int64_t n = 0;
-    for (int b = 0; b < t.batch; ++b) {
-      const int tiles = (t.prompt_len[b] + extra_keys + tile_keys - 1) / tile_keys;
-      n += (tiles + c - 1) / c;
-    }
-    if (n > t.batch + kUmmaMaxChunks) continue;
-    const int64_t waves = (n * n_kv_heads + n_sm - 1) / n_sm;
-    const double cost = (double)waves * (c + 3.0);
-    if (best_c == 0 || cost < best_cost) { best_c = c; best_cost = cost; }
-  }
-  if (best_c == 0) return false;
-  ct->chunk_tiles = best_c;
-  int32_t n = 0;
-  for (int b = 0; b < t.batch; ++b) {
-    const int tiles = (t.prompt_len[b] + extra_keys + tile_keys - 1) / tile_keys;
-    ct->cu_chunk[b] = n;
-    n += (tiles + best_c - 1) / best_c;
-  }
-  ct->cu_chunk[t.batch] = n;
-  ct->n_chunks = n;
-  return true;
-}
-
 }  // namespace
 
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo) {
@@ -120,6 +56,7 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
   if (!plan_chunks(t, dm.n_pseudo, kTile1, dm.n_kv_heads, n_sm, &plan->ct1)) return false;
   if (!plan_chunks(t, 0, kTile2, dm.n_kv_heads, n_sm, &plan->ct2)) return false;
   plan->has_lo = has_lo;
+  plan->lo_sweep1 = plan->lo_sweep2 = has_lo;
   plan->lo_row_offset = lo_row_offset;
   // ---- tensor maps: K as [d, rows, H_kv] (one map per sweep: the boxes differ), the query operand as [d, rows]
   const uint64_t rows_k = (uint64_t)t.cu_rows[t.batch];
@@ -130,8 +67,8 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
   const uint64_t qd[2] = {(uint64_t)kHeadDim, has_lo ? (uint64_t)lo_row_offset + q_rows : q_rows};
   const uint64_t qs[1] = {(uint64_t)kHeadDim * 2};
   if (ks[1] == 0 || ks[1] % 16) return false;
-  return encode_bf16_map(&plan->tm_k1, cv.k, 3, kd, ks, kTile1) && encode_bf16_map(&plan->tm_k2, cv.k, 3, kd, ks, kTile2) &&
-         encode_bf16_map(&plan->tm_q, q_hi, 2, qd, qs, 128);
+  return encode_tile_map(&plan->tm_k1, cv.k, false, 3, kd, ks, kTile1) && encode_tile_map(&plan->tm_k2, cv.k, false, 3, kd, ks, kTile2) &&
+         encode_tile_map(&plan->tm_q, q_hi, false, 2, qd, qs, 128);
 }
 
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
@@ -162,20 +99,23 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
     if ((e = cudaFuncSetAttribute(sweep1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(sweep2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
     if (lse_in == nullptr) {
+      a.has_lo = plan.lo_sweep1;
       log->begin(kKindSweep1, s);
-      launch_pdl(sweep1, dim3(plan.ct1.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k1, plan.tm_q, t,
-                 plan.ct1, a);
+      e = launch_pdl(sweep1, dim3(plan.ct1.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k1, plan.tm_q, t,
+                     plan.ct1, a);
       log->end(s);
+      if (e != cudaSuccess) return e;
     }
+    a.has_lo = plan.lo_sweep2;
     log->begin(kKindSweep2, s);
-    launch_pdl(sweep2, dim3(plan.ct2.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k2, plan.tm_q, t,
-               plan.ct2, plan.ct1, a);
+    e = launch_pdl(sweep2, dim3(plan.ct2.n_chunks, dm.n_kv_heads), dim3(kThreads), kSmemBytes, s, 1, plan.tm_k2, plan.tm_q, t,
+                   plan.ct2, plan.ct1, a);
     log->end(s);
-    return cudaSuccess;
+    return e;
   };
-  const cudaError_t e = !compact      ? run(score_sweep1_kernel<false>, score_sweep2_kernel<false, false>)
-                        : plan.has_lo ? run(score_sweep1_kernel<true>, score_sweep2_kernel<true, true>)
-                                      : run(score_sweep1_kernel<true>, score_sweep2_kernel<true, false>);
+  const cudaError_t e = !compact          ? run(score_sweep1_kernel<false>, score_sweep2_kernel<false, false>)
+                        : plan.lo_sweep2  ? run(score_sweep1_kernel<true>, score_sweep2_kernel<true, true>)
+                                          : run(score_sweep1_kernel<true>, score_sweep2_kernel<true, false>);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }

@@ -34,6 +34,18 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same test, but the thread may be suspended by the hardware for up to ~`ns` nanoseconds while the
+// phase is incomplete (it resumes as soon as the phase completes): a waiting warp then costs the
+// scheduler a few instructions per microsecond instead of a tight polling loop.
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 // Bounded wait of at most `limit` cycles.  Returns false if the CTA is aborting (this or another
 // wait ran out): the caller then leaves its loop, and the CTA drains and returns normally.
 __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
@@ -41,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, v
   if (mbar_try(bar, parity)) return true;
   const long long start = clock64();
   while (true) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try_suspend(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
     if (clock64() - start > limit) {
       *abort_flag = 1;

@@ -52,6 +52,35 @@ def test_rope_matches_transformers_llama():
     np.testing.assert_allclose(mine, lib[0].numpy(), atol=2e-5)
 
 
+def test_llama3_scaled_frequencies_match_transformers_and_the_rule():
+    """rope_inv_freq_llama3 against the library routine for the "llama3" rope type, and against what
+    the rule fixes by itself: fast channels untouched, slow channels divided by the factor, the band
+    in between strictly inside the two, frequencies still decreasing."""
+    ru = pytest.importorskip("transformers.modeling_rope_utils")
+    from transformers import LlamaConfig
+    for d, base, factor, lo, hi, orig in [(128, 5.0e5, 8.0, 1.0, 4.0, 8192), (64, 1.0e4, 32.0, 1.0, 4.0, 8192),
+                                          (128, 1.0e6, 4.0, 2.0, 8.0, 4096)]:
+        cfg = LlamaConfig(hidden_size=4 * d, num_attention_heads=4, head_dim=d, rope_theta=base,
+                          max_position_embeddings=16 * orig,
+                          rope_scaling={"rope_type": "llama3", "factor": factor, "low_freq_factor": lo,
+                                        "high_freq_factor": hi, "original_max_position_embeddings": orig})
+        lib, att = ru.ROPE_INIT_FUNCTIONS["llama3"](cfg, "cpu")
+        mine = orc.rope_inv_freq_llama3(d, base, factor, lo, hi, orig)
+        assert att == 1.0
+        np.testing.assert_allclose(mine, lib.double().numpy(), rtol=2e-6)      # the library works in float32
+        plain = orc.rope_inv_freq(d, base)
+        wl = 2 * np.pi / plain
+        fast, slow = wl < orig / hi, wl > orig / lo
+        assert fast.any() and slow.any() and (~fast & ~slow).any()
+        np.testing.assert_array_equal(mine[fast], plain[fast])
+        np.testing.assert_allclose(mine[slow], plain[slow] / factor, rtol=1e-15)
+        mid = ~fast & ~slow
+        assert np.all(mine[mid] < plain[mid]) and np.all(mine[mid] > plain[mid] / factor)
+        assert np.all(np.diff(mine) < 0)
+    # factor 1 is no scaling at all
+    np.testing.assert_allclose(orc.rope_inv_freq_llama3(128, 5.0e5, 1.0), orc.rope_inv_freq(128, 5.0e5), rtol=1e-15)
+
+
 def test_rope_identity_norm_and_relative_property():
     q, k = _rand((3, 6, 32), 2), _rand((3, 6, 32), 3)
     np.testing.assert_array_equal(orc.rope_pseudo_q(q[:, :1], 0, 1.0e4), q[:, :1])
