@@ -281,13 +281,19 @@ DAPQ_API dapq_status dapq_evict_layers_host(dapq_ctx* ctx, int32_t n_layers, con
  *
  * The scratch of the two sweeps lives in one fixed array of DAPQ_STATIC_SCRATCH_BYTES inside
  * the library image, which every GPU that loads the library holds until the process exits.  A
- * call needs  sum_b (ceil(L_b / 512) + 1) * H_q * N * 8  +  B * H_q * N * 4  bytes of it (e.g.
- * 64k prompt tokens at H_q = 32, N = 64); a larger call returns DAPQ_ERR_WORKSPACE and launches
- * nothing.  All calls on a device share the array: calls whose kernels can overlap on the GPU
- * (different streams, no dependency) race on it and must be ordered by the caller.  Nothing in
- * it needs clearing between calls.  The first call on each device resolves the array's device
- * address (a one-time, per-device set-up with that device current); make that first call
- * outside any stream capture.
+ * call needs  round_up(B * H_q * N * 4, 256)  +  sum_b (ceil(L_b / 512) + 1) * H_q * N * 8  bytes of
+ * it (at H_q = 32, N = 64 a single prompt of up to 64512 tokens fits: 8192 + 127 * 16384 bytes); a
+ * larger call returns DAPQ_ERR_WORKSPACE and launches nothing.  All calls on a device share the
+ * array: calls whose kernels can overlap on the GPU (different streams, no dependency) race on
+ * it and must be ordered by the caller.  Nothing in it needs clearing between calls.
+ *
+ * The FIRST call on each device is a warm-up and is not allocation-free: with that device current
+ * it resolves the array's device address, which makes the CUDA runtime load the module that holds
+ * the array, and it touches every kernel this entry point can launch so that their code is brought
+ * to the device then and not by some later call (the runtime loads a kernel's code at its first
+ * use, and that takes device memory).  Make that first call (any valid small problem will do)
+ * before the point from which the process may no longer allocate, and outside any stream capture.
+ * Every later call on that device, whatever its shape or dtype, allocates nothing.
  * err_out (nullable, host): receives a NUL-terminated reason when the status is not DAPQ_OK. */
 enum { DAPQ_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024 };
 DAPQ_API dapq_status dapq_score_static(const dapq_shape* shape, int device, const void* q_rot,

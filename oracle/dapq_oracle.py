@@ -156,6 +156,33 @@ def score_sequence(q_rot: np.ndarray, k_seq: np.ndarray, prompt_len: int, group:
     return {"scores": scores, "lse": lse, "prompt_mass": pm, "syn_mass": sm}
 
 
+def score_prompt_window(q_win_rot: np.ndarray, k_seq: np.ndarray, group: int,
+                        scale: Optional[float] = None) -> np.ndarray:
+    """Scores of the SnapKV-style observation window the paper compares against (Section 5.1): the
+    N queries are those of the LAST N prompt tokens (already rotated), window query i sits at
+    position L - N + i and, under the causal mask, attends to keys 0 .. L - N + i.
+
+    q_win_rot [H_q, N, d]; k_seq [H_kv, L, d] (the whole prompt, no synthetic rows).  Returns
+    [H_kv, L - N]: sum over the window queries and the group's heads of the attention each token
+    BEFORE the window receives (the window's own tokens are always kept by that method).
+    """
+    q = np.asarray(q_win_rot, dtype=np.float64)
+    kk = np.asarray(k_seq, dtype=np.float64)
+    Hq, n, d = q.shape
+    Hkv, L, _ = kk.shape
+    sc = 1.0 / math.sqrt(d) if scale is None else float(scale)
+    out = np.zeros((Hkv, L - n), dtype=np.float64)
+    key_pos = np.arange(L)[None, :]
+    query_pos = (L - n + np.arange(n))[:, None]
+    for h in range(Hq):
+        s = (q[h] @ kk[h // group].T) * sc                      # [N, L]
+        s = np.where(key_pos <= query_pos, s, -np.inf)
+        e = np.exp(s - s.max(axis=1, keepdims=True))
+        P = e / e.sum(axis=1, keepdims=True)
+        out[h // group] += P[:, :L - n].sum(axis=0)
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # Optional pooling of the accumulated scores before selection.  The paper specifies none
 # for DapQ; it describes the SnapKV / PyramidKV baselines as selecting on pooled accumulated

@@ -167,9 +167,13 @@ dapq_status build_table(dapq_ctx* ctx, int32_t batch, const int32_t* cu_rows, co
   t->cu_prompt[batch] = (int32_t)prompt;
   t->cu_keep[batch] = (int32_t)keep;
   const int64_t last_row = cu_rows ? cu_rows[batch] : rows;
-  if ((prompt_len || cu_prompt) && (last_row > sh.max_total_rows || chunks > ctx->max_chunks))
+  if ((prompt_len || cu_prompt) && last_row > sh.max_total_rows)
     return fail(ctx, DAPQ_ERR_WORKSPACE, "%lld cache rows exceed max_total_rows %lld",
                 (long long)last_row, (long long)sh.max_total_rows);
+  if ((prompt_len || cu_prompt) && chunks > ctx->max_chunks)
+    return fail(ctx, DAPQ_ERR_WORKSPACE, "%lld work chunks of %d keys exceed the %lld the workspace was sized for "
+                "(more or longer sequences than max_batch / max_total_rows allow)",
+                (long long)chunks, kChunkKeys, (long long)ctx->max_chunks);
   return DAPQ_OK;
 }
 
@@ -640,11 +644,36 @@ const void* mapped_v(dapq_ctx* ctx, const CacheDev& hv) {
 
 }  // namespace
 
+namespace {
+dapq_status evict_layers_host_impl(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre_host,
+                                   const dapq_cache_view* caches_host, const int32_t* k_keep_host,
+                                   int64_t k_keep_layer_stride, void* const* k_out_host, void* const* v_out_host,
+                                   int32_t* const* idx_out_host, void* stream);
+}  // namespace
+
 dapq_status dapq_evict_layers_host(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre_host,
                                    const dapq_cache_view* caches_host, const int32_t* k_keep_host,
                                    int64_t k_keep_layer_stride, void* const* k_out_host, void* const* v_out_host,
                                    int32_t* const* idx_out_host, void* stream) {
   if (!ctx) return DAPQ_ERR_INVALID_ARG;
+  const dapq_status st = evict_layers_host_impl(ctx, n_layers, q_pre_host, caches_host, k_keep_host, k_keep_layer_stride,
+                                                k_out_host, v_out_host, idx_out_host, stream);
+  if (st != DAPQ_OK) {
+    // a layer failed with copies of earlier layers possibly still in flight: the caller's buffers may be
+    // reused as soon as this call returns, so wait for both streams first (their own errors do not matter now)
+    DeviceGuard guard(ctx->device);
+    if (ctx->copy_stream) cudaStreamSynchronize(ctx->copy_stream);
+    cudaStreamSynchronize((cudaStream_t)stream);
+    cudaGetLastError();
+  }
+  return st;
+}
+
+namespace {
+dapq_status evict_layers_host_impl(dapq_ctx* ctx, int32_t n_layers, const void* const* q_pre_host,
+                                   const dapq_cache_view* caches_host, const int32_t* k_keep_host,
+                                   int64_t k_keep_layer_stride, void* const* k_out_host, void* const* v_out_host,
+                                   int32_t* const* idx_out_host, void* stream) {
   if (n_layers < 0 || k_keep_layer_stride < 0) return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers_host: negative count or stride");
   if (n_layers > 0 && (!q_pre_host || !caches_host || !k_keep_host || !k_out_host || !v_out_host))
     return fail(ctx, DAPQ_ERR_INVALID_ARG, "dapq_evict_layers_host: NULL argument");
@@ -724,6 +753,7 @@ dapq_status dapq_evict_layers_host(dapq_ctx* ctx, int32_t n_layers, const void* 
   DAPQ_CUDA(ctx, cudaStreamSynchronize(s));
   return DAPQ_OK;
 }
+}  // namespace
 
 dapq_status dapq_evict_host(dapq_ctx* ctx, const void* q_pre_host, const dapq_cache_view* cache_host,
                             const int32_t* k_keep_host, void* k_out_host, void* v_out_host,

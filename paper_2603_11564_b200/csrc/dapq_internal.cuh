@@ -135,6 +135,9 @@ cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const Ca
                              float* lse2, float* scores, int64_t score_stride, float* lse_out, float* syn_mass,
                              cudaStream_t s, LaunchLog* log);
 
+// Makes the device code of every CUDA-core score kernel resident on the current device (no launch).
+cudaError_t score_fma_preload();
+
 // Tensor-core scorer (bf16 caches).  umma_plan encodes the TMA descriptors and cuts the work;
 // it returns false when the view cannot be described to TMA (the caller then takes the
 // CUDA-core path).  q_hi: [B*H_q*N, d] bf16; with has_lo the low-order parts follow

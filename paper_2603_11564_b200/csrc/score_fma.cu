@@ -322,6 +322,36 @@ cudaError_t run_fma_n(const void* q_rot, const CacheDev& cv, const SeqTable& t, 
 
 }  // namespace
 
+namespace {
+template <typename TQ, typename T, int R>
+cudaError_t preload_fma() {
+  constexpr size_t smem = fma_smem_bytes<R>();
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(score_fma_kernel<TQ, T, R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(score_fma_kernel<TQ, T, R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+template <typename TQ, typename T>
+cudaError_t preload_fma_n() {
+  cudaError_t e;
+  if ((e = preload_fma<TQ, T, 1>()) != cudaSuccess) return e;
+  if ((e = preload_fma<TQ, T, 2>()) != cudaSuccess) return e;
+  if ((e = preload_fma<TQ, T, 4>()) != cudaSuccess) return e;
+  return preload_fma<TQ, T, 8>();
+}
+}  // namespace
+
+// Touch every kernel that launch_score_fma can pick for storage type == query type, so that the device
+// code of all of them is resident on the current device afterwards (with lazy module loading a kernel's
+// code is brought to the device, and device memory taken for it, at its first use).
+cudaError_t score_fma_preload() {
+  cudaError_t e;
+  if ((e = preload_fma_n<__nv_bfloat16, __nv_bfloat16>()) != cudaSuccess) return e;
+  if ((e = preload_fma_n<float, float>()) != cudaSuccess) return e;
+  cudaFuncAttributes fa;
+  if ((e = cudaFuncGetAttributes(&fa, lse_merge_kernel)) != cudaSuccess) return e;
+  return cudaFuncGetAttributes(&fa, lse_import_kernel);
+}
+
 cudaError_t launch_score_fma(int dtype, int q_dtype, const void* q_rot, const CacheDev& cv, const SeqTable& t,
                              const Dims& dm, const float* lse_in, float2* part, int64_t max_chunks, int n_sm,
                              float* lse2, float* scores, int64_t score_stride, float* lse_out, float* syn_mass,

@@ -103,7 +103,8 @@ extern "C" dapq_status dapq_score_static(const dapq_shape* sh, int device, const
   if (need > (size_t)DAPQ_STATIC_SCRATCH_BYTES)
     return fail_static(err, err_len, DAPQ_ERR_WORKSPACE,
                        "dapq_score_static: this call needs %zu bytes of scratch, the fixed area holds %d "
-                       "(chunks of 512 keys x H_q x N x 8 bytes); use dapq_create + dapq_score for larger caches",
+                       "(round_up(B x H_q x N x 4, 256) + sum_b (ceil(L_b / 512) + 1) x H_q x N x 8 bytes); use "
+                       "dapq_create + dapq_score for larger caches",
                        need, (int)DAPQ_STATIC_SCRATCH_BYTES);
   // what is left lets the launcher cut small inputs into finer chunks
   const int64_t max_chunks = (int64_t)(((size_t)DAPQ_STATIC_SCRATCH_BYTES - part_off) / (hq_n * sizeof(float2)));
@@ -112,13 +113,19 @@ extern "C" dapq_status dapq_score_static(const dapq_shape* sh, int device, const
   if (!scope.ok) return fail_static(err, err_len, DAPQ_ERR_CUDA, "cannot make device %d current", device);
   void* base = nullptr;
   {
-    // set-up, once per device, with that device current: resolve the array's device address
+    // set-up, once per device, with that device current: resolve the array's device address (this loads the
+    // module that holds the array)
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_scratch_addr[device]) {
       void* p = nullptr;
       const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
       if (e != cudaSuccess || !p)
         return fail_static(err, err_len, DAPQ_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+      // ... and bring the code of every kernel this entry point can launch to the device now, so that no later
+      // call has to (a kernel's first use loads its code, which takes device memory)
+      const cudaError_t e2 = score_fma_preload();
+      if (e2 != cudaSuccess)
+        return fail_static(err, err_len, DAPQ_ERR_CUDA, "loading the score kernels: %s", cudaGetErrorString(e2));
       g_scratch_addr[device] = p;
     }
     base = g_scratch_addr[device];

@@ -53,13 +53,15 @@ __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, v
   if (mbar_try(bar, parity)) return true;
   const long long start = clock64();
   while (true) {
-    if (mbar_try_suspend(bar, parity, 20000u)) return true;
-    if (*abort_flag) return false;
+    // (the clock is read before the suspended try, so that a limit of a few cycles gives up on the first wait
+    // that is not satisfied at once, whatever the suspension hides)
     if (clock64() - start > limit) {
       *abort_flag = 1;
       atomicOr(status, kStatusTimeout);
       return false;
     }
+    if (mbar_try_suspend(bar, parity, 20000u)) return true;
+    if (*abort_flag) return false;
   }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
@@ -91,6 +93,10 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+// Ask L2 for a tile (nothing lands in shared memory, no barrier is involved).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int x, int y, int z) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }

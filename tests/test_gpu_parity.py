@@ -246,15 +246,58 @@ def test_evict_tiny_config_in_full(dq):
     _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
 
 
-@pytest.mark.parametrize("cuda_core", [False, True])
+SCORERS = {"fp16": 0, "cuda_core": 1, "bf16_pair": 8 | 16}   # dapq_shape.flags
+
+
+@pytest.mark.parametrize("scorer", list(SCORERS))
 @pytest.mark.parametrize("name,scale", [("llama3_8b_32k", 16), ("qwen25_7b_128k", 64), ("batched_serving", 16),
                                         ("llama3_70b_128k", 64)])
-def test_evict_scaled_configs(dq, name, scale, cuda_core):
+def test_evict_scaled_configs(dq, name, scale, scorer):
+    """Every scorer the flags select (default fp16 tensor-core path, CUDA cores, the older tensor-core kernels
+    with the two-part bf16 query operand in both sweeps) meets the same criteria."""
     w = gi.scaled_down(name, scale, n_layers=1)
     data = util.make_case(w)
-    ctx = _ctx(dq, w, flags=dq.DAPQ_FLAG_CUDA_CORE_SCORER if cuda_core else 0)
+    ctx = _ctx(dq, w, flags=SCORERS[scorer])
     _check_evict(w, data, _gpu_evict(dq, w, data, ctx), util.oracle_evict(w, data))
     dq.dapq_destroy(ctx)
+
+
+def test_coarse_query_modes_are_close_but_worse_than_the_default(dq):
+    """DAPQ_FLAG_Q_BF16 (one bf16 rounding of the rotated queries) and the two-part operand in one sweep only are
+    the documented coarse modes: on a cache with outlier channels their scores stay within 2e-2 of the oracle
+    but are measurably worse than the default's."""
+    w = gi.scaled_down("llama3_8b_32k", 8, n_layers=1)
+    data = util.make_case(w)
+    ref = util.oracle_evict(w, data)["scores"][0]
+    worst = {}
+    for name, flags in (("fp16", 0), ("bf16", dq.DAPQ_FLAG_Q_BF16), ("pair_sweep1", dq.DAPQ_FLAG_Q_LO_SWEEP1),
+                        ("pair_sweep2", dq.DAPQ_FLAG_Q_LO_SWEEP2)):
+        ctx = _ctx(dq, w, flags=flags)
+        got = _gpu_evict(dq, w, data, ctx)["scores"]
+        dq.dapq_destroy(ctx)
+        worst[name] = float(np.max(np.abs(got - ref) / ref))
+    assert worst["fp16"] < 1e-3, worst
+    for name in ("bf16", "pair_sweep1", "pair_sweep2"):
+        assert worst["fp16"] < worst[name] < 2e-2, worst
+
+
+def test_score_with_the_older_kernels(dq):
+    """A context that asks for the two-part operand sends dapq_score (whose bf16 queries have no low-order
+    part) through the older tensor-core kernels as well; several query groups, ragged lengths."""
+    for hq, hkv, n, lens in [(8, 1, 128, (129, 1031)), (8, 2, 64, (1500,)), (4, 4, 32, (700, 64))]:
+        w = _small(lens=lens, keep=tuple(1 for _ in lens), n_q_heads=hq, n_kv_heads=hkv, n_pseudo=n, n_needles=0,
+                   outlier_channels=2)
+        data = gi.draw_layer(w, 0, "cpu")
+        q_rot = util.oracle_q_rot(w, data).to(torch.bfloat16)
+        ctx = _ctx(dq, w, flags=dq.DAPQ_FLAG_Q_LO_SWEEP1 | dq.DAPQ_FLAG_Q_LO_SWEEP2)
+        scores = torch.empty((hkv, w.total_prompt), dtype=torch.float32, device="cuda")
+        dq.dapq_score(ctx, q_rot.cuda(), data["k"].cuda(), w.cu_rows, w.prompt_lens, scores)
+        dq.dapq_poll_status(ctx)
+        dq.dapq_destroy(ctx)
+        got, k64 = scores.cpu().double().numpy(), util.to_f64(data["k"])
+        for b in range(w.batch):
+            ref = orc.score_sequence(util.to_f64(q_rot[b]), k64[:, int(w.cu_rows[b]):int(w.cu_rows[b + 1])], lens[b], w.group)
+            util.assert_scores_close(got[:, w.cu_prompt[b]:w.cu_prompt[b + 1]], ref["scores"], f"older kernels b={b}")
 
 
 def test_evict_edge_shapes(dq):
@@ -551,21 +594,13 @@ def test_evict_layers_replays_from_a_cuda_graph(dq):
 def test_prompt_window_variant_uses_the_same_entry_points(dq):
     """The SnapKV-style window of Section 5.1's baselines (queries = the last N prompt tokens, query i sees
     keys up to its own position, window rows always kept) is the same computation with prompt_len = L - N:
-    the window's rows play the part of the synthetic rows.  Reference: the causal attention matrix written
-    out with torch in float64."""
+    the window's rows play the part of the synthetic rows.  Reference: the oracle's score_prompt_window."""
     L, N, hq, hkv, keep = 1500, 32, 8, 2, 200
     w = _small(lens=(L - N,), keep=(keep - N,), n_q_heads=hq, n_kv_heads=hkv, n_pseudo=N, n_needles=0)
     data = gi.draw_layer(w, 0, "cpu")                            # k: [H_kv, L, d]; q_pre stands for the window's rotated queries
     q_win, k = data["q_pre"], data["k"]
     assert k.shape[1] == L
-    qd, kd = q_win[0].double(), k.double()
-    pos_q = torch.arange(L - N, L).view(N, 1)
-    visible = torch.arange(L).view(1, L) <= pos_q                 # causal: key j <= position of window query i
-    ref = torch.zeros(hkv, L - N, dtype=torch.float64)
-    for h in range(hq):
-        logits = (qd[h] @ kd[h // (hq // hkv)].T) / np.sqrt(128.0)
-        probs = torch.softmax(logits.masked_fill(~visible, float("-inf")), dim=-1)
-        ref[h // (hq // hkv)] += probs[:, :L - N].sum(0)
+    ref = torch.from_numpy(orc.score_prompt_window(util.to_f64(q_win[0]), util.to_f64(k), hq // hkv))
     ctx = _ctx(dq, w)
     scores = torch.empty((hkv, L - N), dtype=torch.float32, device="cuda")
     dq.dapq_score(ctx, q_win.cuda(), k.cuda(), w.cu_rows, w.prompt_lens, scores)
@@ -615,3 +650,108 @@ def test_evict_largest_batch(dq):
     w = _small(lens=lens, keep=keep, n_q_heads=8, n_kv_heads=2, n_pseudo=16, n_needles=0)
     data = gi.draw_layer(w, 0, "cpu")
     _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+
+
+# ----------------------------------------------------------------- precision of the query operand
+@pytest.mark.parametrize("name,heads,bound", [("llama3_8b_32k", (0, 3), 1e-3), ("llama3_70b_128k", (6,), 1e-3)])
+def test_default_precision_full_size_within_half_the_budget(dq, name, heads, bound):
+    """The default query precision (fp16, K converted on the fly) keeps the worst per-token error of the two
+    configurations with outlier channels, at full size, below 1e-3: half of the 2e-3 budget."""
+    w = gi.workload(name)
+    data = gi.draw_layer(w, 0, "cuda")
+    ctx = _ctx(dq, w)
+    q_rot = torch.empty_like(data["q_pre"])
+    dq.dapq_rope_pseudo_q(ctx, data["q_pre"], list(w.prompt_lens), q_rot)
+    torch.cuda.synchronize()
+    gi.plant_structure(w, data, q_rot)
+    got = _gpu_evict(dq, w, data, ctx)["scores"]
+    dq.dapq_destroy(ctx)
+    G, N, L = w.group, w.n_pseudo, w.prompt_lens[0]
+    q64 = util.to_f64(data["q_pre"])
+    for h in heads:
+        qr = orc.rope_pseudo_q(q64[0, h * G:(h + 1) * G], L, w.rope_base)
+        ref = orc.score_sequence(qr, util.to_f64(data["k"][h].cpu())[None, :L + N], L, G)["scores"][0]
+        worst = float(np.max(np.abs(got[h] - ref) / ref))
+        assert worst < bound, f"{name} kvh={h}: worst relative error {worst:.3e}"
+
+
+# ----------------------------------------------------------------------- Llama-3.1 scaled RoPE
+def test_evict_with_llama31_rope_preset(dq):
+    """The frequency table of Llama-3.1's long-context scaling (the model of the paper's efficiency runs),
+    produced by the library's helper, through the whole path; the oracle rotates with its own statement
+    of the same rule."""
+    w = _small(lens=(1200, 410), keep=(60, 25), n_q_heads=8, n_kv_heads=2, n_pseudo=32, n_needles=0, rope_base=5.0e5)
+    inv = np.array(dq.dapq_rope_inv_freq_llama3(5.0e5, 8.0, 1.0, 4.0, 8192))
+    ref_inv = orc.rope_inv_freq_llama3(128, 5.0e5, 8.0, 1.0, 4.0, 8192)
+    np.testing.assert_allclose(inv, ref_inv, rtol=1e-14)
+    data = gi.draw_layer(w, 0, "cpu")
+    ref = orc.evict(util.to_f64(data["q_pre"]), util.to_f64(data["k"]), util.to_f64(data["v"]), w.cu_rows,
+                    w.prompt_lens, w.keep, w.rope_base, inv_freq=ref_inv)
+    assert not np.allclose(ref["scores"][0], util.oracle_evict(w, data)["scores"][0], rtol=1e-3)   # the scaling matters
+    for flags in (0, dq.DAPQ_FLAG_CUDA_CORE_SCORER):
+        ctx = _ctx(dq, w, inv_freq=list(inv), flags=flags)
+        _check_evict(w, data, _gpu_evict(dq, w, data, ctx), ref)
+        dq.dapq_destroy(ctx)
+
+
+# ------------------------------------------------------------ the call the benchmark times, at full size
+def test_evict_layers_full_size_sampled_heads(dq):
+    """Two layers of the Llama-3-8B-shaped cache at full size through dapq_evict_layers (the call bench.py
+    steps through), sampled KV heads against the oracle."""
+    w = gi.workload("llama3_8b_32k")
+    ctx = _ctx(dq, w)
+    datas = []
+    for l in range(2):
+        d = gi.draw_layer(w, l, "cuda")
+        q_rot = torch.empty_like(d["q_pre"])
+        dq.dapq_rope_pseudo_q(ctx, d["q_pre"], list(w.prompt_lens), q_rot)
+        torch.cuda.synchronize()
+        gi.plant_structure(w, d, q_rot)
+        datas.append(d)
+    KT, L, G, N = int(w.cu_keep[-1]), w.prompt_lens[0], w.group, w.n_pseudo
+    ko = [torch.empty((w.n_kv_heads, KT, 128), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    vo = [torch.empty_like(t) for t in ko]
+    idx = [torch.empty((w.n_kv_heads, KT), dtype=torch.int32, device="cuda") for _ in range(2)]
+    dq.dapq_evict_layers(ctx, [d["q_pre"] for d in datas], [d["k"] for d in datas], [d["v"] for d in datas], w.cu_rows,
+                         w.prompt_lens, w.keep, ko, vo, idx)
+    dq.dapq_poll_status(ctx)
+    dq.dapq_destroy(ctx)
+    for l, h in ((0, 2), (1, 5)):
+        d = datas[l]
+        k_h, v_h = d["k"][h].cpu(), d["v"][h].cpu()
+        qr = orc.rope_pseudo_q(util.to_f64(d["q_pre"])[0, h * G:(h + 1) * G], L, w.rope_base)
+        ref = orc.score_sequence(qr, util.to_f64(k_h)[None, :L + N], L, G)["scores"][0]
+        gidx = idx[l][h].cpu().numpy()
+        util.assert_index_sets_match(gidx, ref, orc.topk_select(ref, w.keep[0]), L, f"layer {l} kvh={h}")
+        rows = torch.as_tensor(gidx.astype(np.int64))
+        assert torch.equal(ko[l][h].cpu(), k_h[rows]) and torch.equal(vo[l][h].cpu(), v_h[rows])
+        for p in d["needle_pos"][0, h]:
+            assert int(p) in set(gidx.tolist())
+
+
+# ------------------------------------------------------------------ a device-side wait that runs out
+def test_wait_limit_gives_up_reports_timeout_and_recovers(dq):
+    """With the wait bound set to one cycle, the first wait of every score CTA that is not satisfied at once
+    runs out: the kernels return normally, dapq_poll_status reports DAPQ_ERR_TIMEOUT once and clears the
+    status word, and the same context then computes the right answer again."""
+    w = gi.scaled_down("llama3_8b_32k", 8, n_layers=1)
+    data = util.make_case(w)
+    ref = util.oracle_evict(w, data)
+    ctx = _ctx(dq, w)
+    good = _gpu_evict(dq, w, data, ctx)
+    dq.dapq_set_wait_limit(ctx, 1)
+    q, k, v = (data[x].cuda() for x in ("q_pre", "k", "v"))
+    KT = int(w.cu_keep[-1])
+    k_out = torch.empty((w.n_kv_heads, KT, 128), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    dq.dapq_evict(ctx, q, k, v, w.cu_rows, w.prompt_lens, w.keep, k_out, v_out)
+    with pytest.raises(dq.DapqError) as e:
+        dq.dapq_poll_status(ctx)
+    assert e.value.status == dq.DAPQ_ERR_TIMEOUT
+    dq.dapq_poll_status(ctx)                                     # the word was cleared by the poll above
+    dq.dapq_set_wait_limit(ctx, 0)
+    again = _gpu_evict(dq, w, data, ctx)
+    np.testing.assert_array_equal(again["scores"], good["scores"])
+    np.testing.assert_array_equal(again["idx"], good["idx"])
+    _check_evict(w, data, again, ref)
+    dq.dapq_destroy(ctx)

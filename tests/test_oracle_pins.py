@@ -416,3 +416,31 @@ def test_recall_of_a_smaller_window_against_a_larger_one():
     pred = orc.evict(q[:, :, 12:], k4, k4, [0, 64], [60], [10], 1.0e4, pos_start=[72])["idx"][0][0]
     r = orc.recall(gold, pred)
     assert 0.0 <= r <= 1.0 and abs(r * 10 - round(r * 10)) < 1e-12
+
+
+def test_prompt_window_scores_match_library_causal_attention():
+    """score_prompt_window against torch's scaled_dot_product_attention over the L-token prompt (value
+    matrix = identity, so the output rows ARE the attention weights), and against the identity that
+    ties it to the pseudo-query scorer: a window cut from the prompt is the same computation with
+    prompt_len = L - N and the window's rows in the place of the synthetic rows."""
+    rng = np.random.default_rng(5)
+    for Hq, Hkv, n, L, d in [(4, 2, 3, 17, 8), (2, 2, 5, 40, 16), (6, 2, 1, 9, 4)]:
+        G = Hq // Hkv
+        q = rng.standard_normal((Hq, n, d))
+        k = rng.standard_normal((Hkv, L, d))
+        got = orc.score_prompt_window(q, k, G)
+        qt, kt = torch.from_numpy(q), torch.from_numpy(k).repeat_interleave(G, dim=0)
+        mask = torch.arange(L)[None, :] <= (L - n + torch.arange(n))[:, None]
+        P = torch.nn.functional.scaled_dot_product_attention(qt[None], kt[None], torch.eye(L, dtype=torch.float64).expand(1, Hq, L, L),
+                                                             attn_mask=mask)[0]
+        want = P[:, :, :L - n].sum(dim=1).reshape(Hkv, G, L - n).sum(dim=1).numpy()
+        np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(got, orc.score_sequence(q, k, L - n, G)["scores"], rtol=1e-12, atol=1e-15)
+    # a planted mistake (strictly causal window: a query that does not see its own key) fails the pin
+    q, k = rng.standard_normal((2, 3, 8)), rng.standard_normal((1, 12, 8))
+    good = orc.score_prompt_window(q, k, 2)
+    s = np.einsum("hnd,ld->hnl", q, k[0]) / np.sqrt(8.0)
+    s = np.where(np.arange(12)[None, None, :] < (9 + np.arange(3))[None, :, None], s, -np.inf)
+    e = np.exp(s - s.max(-1, keepdims=True))
+    bad = (e / e.sum(-1, keepdims=True))[:, :, :9].sum(axis=(0, 1))
+    assert not np.allclose(good[0], bad, rtol=1e-3)
