@@ -28,7 +28,8 @@ template <> __device__ __forceinline__ float from_double<float>(double x) { retu
 template <> __device__ __forceinline__ __nv_bfloat16 from_double<__nv_bfloat16>(double x) {
   return __double2bfloat16(x);
 }
-// fp16 output (the query operand of the fp16 MMAs): values beyond the format's range saturate
+// fp16 output (the query operand of the fp16 MMAs, stored times softmax scale * log2(e) so that the MMAs yield
+// base-2 logits): values beyond the format's range saturate
 template <> __device__ __forceinline__ __half from_double<__half>(double x) {
   return __double2half(fmin(fmax(x, -65504.0), 65504.0));
 }
@@ -39,7 +40,7 @@ __global__ void __launch_bounds__(kHeadDim / 2 * kHeadsPerBlock)
 rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
                      const double* __restrict__ inv_freq, const __grid_constant__ SeqTable t,
                      int n_q_heads, int n_pseudo, int64_t lo_offset, int late_wait,
-                     int interleaved) {
+                     int interleaved, double out_scale) {
   // late_wait: the kernel before this one in the stream neither writes q_pre nor still reads q_rot
   // (it is the compaction of the layer before), so the rotation runs beside it; the wait at the end
   // keeps this grid, and with it everything launched after it, ordered behind that kernel.
@@ -59,7 +60,7 @@ rope_pseudo_q_kernel(const T* __restrict__ q_pre, TO* __restrict__ q_rot,
   const double ang = (double)(t.pos_start[b] + i) * inv_freq[c];
   double sn, cs;
   sincos(ang, &sn, &cs);
-  const double r0 = lo * cs - hi * sn, r1 = hi * cs + lo * sn;
+  const double r0 = (lo * cs - hi * sn) * out_scale, r1 = (hi * cs + lo * sn) * out_scale;
   const TO h0 = from_double<TO>(r0), h1 = from_double<TO>(r1);
   q_rot[e0] = h0;
   q_rot[e1] = h1;
@@ -81,19 +82,19 @@ cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* 
   dim3 block(kHeadDim / 2, kHeadsPerBlock);
   if (dtype == DAPQ_BF16 && out_mode == kRopeOutSplitBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, true>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw, dm.rope_interleaved);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, lo_offset, lw, dm.rope_interleaved, 1.0);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutF16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __half, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__half*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
+               (__half*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved, (double)dm.scale_log2e);
   } else if (dtype == DAPQ_BF16 && out_mode == kRopeOutBf16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, __nv_bfloat16, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
+               (__nv_bfloat16*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved, 1.0);
   } else if (dtype == DAPQ_BF16) {
     launch_pdl(rope_pseudo_q_kernel<__nv_bfloat16, float, false>, grid, block, 0, s, 1, (const __nv_bfloat16*)q_pre,
-               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
+               (float*)q_rot, inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved, 1.0);
   } else {
     launch_pdl(rope_pseudo_q_kernel<float, float, false>, grid, block, 0, s, 1, (const float*)q_pre, (float*)q_rot,
-               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved);
+               inv_freq_dev, t, dm.n_q_heads, dm.n_pseudo, 0, lw, dm.rope_interleaved, 1.0);
   }
   log->end(s);
   return cudaGetLastError();

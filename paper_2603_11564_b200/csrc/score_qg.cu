@@ -128,7 +128,8 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
   plan->rows_g = (((rows_total + plan->n_qgroups - 1) / plan->n_qgroups) + 15) & ~15;
   plan->q_is_f16 = q_is_f16;
   const int q_bytes = ((plan->rows_g + 127) / 128) * 2 * 128 * 128;
-  const int s1 = (kRingEnd - q_bytes) / TileGeo<kTile1>::kStage, s2 = (kRingEnd - q_bytes) / TileGeo<kTile2>::kStage;
+  const int s1 = (kRingEnd - q_bytes) / TileGeo<kTile1>::kStage;
+  const int s2 = (kRingEnd - (q_is_f16 ? kSlabBytes : 0) - q_bytes) / TileGeo<kTile2>::kStage;   // (the -lse operands sit at the end)
   plan->n_stages1 = s1 < kMaxStages ? s1 : kMaxStages;
   plan->n_stages2 = s2 < kMaxStages ? s2 : kMaxStages;
   const int ctas = dm.n_kv_heads * plan->n_qgroups;
@@ -159,7 +160,7 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
   a.n_qgroups = plan.n_qgroups;
   a.rows_g = plan.rows_g;
   a.rows_pad = (a.rows_total + 255) / 256 * 256;
-  a.scale_log2e = dm.scale_log2e;
+  a.scale_log2e = plan.q_is_f16 ? 1.f : dm.scale_log2e;        // the library's own fp16 queries are stored times scale * log2(e)
   a.wait_limit = wait_limit > 0 ? wait_limit : kWaitLimit;
   a.part = part;
   a.lse_in = lse_in;

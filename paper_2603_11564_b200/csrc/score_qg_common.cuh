@@ -33,6 +33,11 @@ constexpr int kMaxStages = DAPQ_MAX_STAGES, kMaxAcc = 4;
 constexpr int kL2Ahead = DAPQ_L2_AHEAD;        // tiles beyond the ring that the producer asks L2 for (0: none)
 constexpr int kExchDepth = 4;                  // jobs whose partial sums can wait in shared memory (sweep 2)
 constexpr int kRingEnd = 216 * 1024;           // queries + K ring end here; the small state follows
+// Sweep 2 with its own fp16 queries appends one k-step to every job's MMAs that adds -lse_i to column i of
+// the accumulator: a [256 x 16] operand holding -lse as an fp16 pair, against a [128 x 16] operand of ones.
+constexpr int kLseSlabBytes = kGroupRows * 32, kOnesSlabBytes = kTile2 * 32;
+constexpr int kSlabBytes = kLseSlabBytes + kOnesSlabBytes;                      // kept at the end of the ring area
+constexpr int kLseSlab = kRingEnd - kSlabBytes, kOnesSlab = kRingEnd - kOnesSlabBytes;
 
 template <int kTile>
 struct TileGeo {
@@ -43,9 +48,9 @@ struct TileGeo {
 // Shared memory behind the ring (offsets from the 1024-aligned base).
 struct Smem {
   static constexpr int bars = kRingEnd;
-  // barriers: k_full[4], k_conv[4], k_empty[4], acc_full[4], acc_empty[4], part_full[4], part_empty[4], q_full, drain
-  static constexpr int n_bars = 3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 2;
-  static constexpr int lse = bars + n_bars * 8;                    // [256] floats (sweep 2); with the next block:
+  // barriers: k_full[4], k_conv[4], k_empty[4], acc_full[4], acc_empty[4], part_full[4], part_empty[4], q_full, drain, lse_ready
+  static constexpr int n_bars = 3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 3;
+  static constexpr int lse = (bars + n_bars * 8 + 15) & ~15;       // [256] floats, read as float4 (sweep 2); with the next block:
                                                                    // [256] float2 row statistics (sweep 1)
   static constexpr int aux = lse + kGroupRows * 4;                 // [256] floats: the other half of the statistics
   static constexpr int exch = aux + kGroupRows * 4;                // [kExchDepth][4][128] floats (sweep 2)
@@ -53,6 +58,7 @@ struct Smem {
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
+static_assert(Smem::lse % 16 == 0 && Smem::aux % 16 == 0 && Smem::exch % 16 == 0, "vector loads need 16-byte alignment");
 constexpr int kSmemBytes = Smem::total;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
@@ -109,6 +115,7 @@ struct Bars {
   }
   __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth); }
   __device__ __forceinline__ uint32_t drain() const { return base + 8u * (3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 1); }
+  __device__ __forceinline__ uint32_t lse_ready() const { return base + 8u * (3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 2); }
 };
 
 // Position in a ring of n slots walked once per tile or job: slot index and the parity of its phase.
@@ -154,6 +161,7 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
     }
     mbar_init(bars.q_full(), 1);
     mbar_init(bars.drain(), 1);
+    mbar_init(bars.lse_ready(), 1);
     *reinterpret_cast<volatile int*>(smem + Smem::abort_flag) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }

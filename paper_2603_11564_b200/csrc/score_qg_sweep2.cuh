@@ -20,29 +20,36 @@ namespace dapq {
 namespace qg {
 
 // 16 accumulator columns of one key row: sum of 2^(s c - lse) over the columns, as two packed pairs.
-// kFull: all 16 columns exist (no per-column test).
-template <bool kFull>
+// kFull: all 16 columns exist (no per-column test).  kFold: the accumulator already holds s c - lse (the
+// queries were scaled before the MMAs and -lse was added by the job's last k-step).
+template <bool kFull, bool kFold>
 __device__ __forceinline__ void colsum_piece(const uint32_t* v, const float* lse16, int valid, float c, float2& acc, float2& acc1) {
   if (kFull) {
     const float2 c2 = make_float2(c, c);
 #pragma unroll
     for (int e = 0; e < 16; e += 4) {
-      const float4 l4 = *reinterpret_cast<const float4*>(lse16 + e);
-      const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2, make_float2(l4.x, l4.y));
-      const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2, make_float2(l4.z, l4.w));
+      float2 x0, x1;
+      if (kFold) {
+        x0 = make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+        x1 = make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+      } else {
+        const float4 l4 = *reinterpret_cast<const float4*>(lse16 + e);
+        x0 = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2, make_float2(l4.x, l4.y));
+        x1 = __ffma2_rn(make_float2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])), c2, make_float2(l4.z, l4.w));
+      }
       acc = __fadd2_rn(acc, ((kPolyPairMask >> (e / 2)) & 1u) ? ex2_pair_poly(x0) : ex2_pair_mufu(x0));
       acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> (e / 2 + 1)) & 1u) ? ex2_pair_poly(x1) : ex2_pair_mufu(x1));
     }
   } else {
 #pragma unroll
     for (int e = 0; e < 16; ++e)
-      if (e < valid) acc.x += ex2(fmaf(__uint_as_float(v[e]), c, lse16[e]));
+      if (e < valid) acc.x += kFold ? ex2(__uint_as_float(v[e])) : ex2(fmaf(__uint_as_float(v[e]), c, lse16[e]));
   }
 }
 
 // This warp's pieces [p0, p0 + np) of one accumulator (np <= 4), two at a time; `release` gives the
 // accumulator back once the last piece is in registers.  kFull: every column of these pieces exists.
-template <bool kFull, class Release>
+template <bool kFull, bool kFold, class Release>
 __device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, int p0, int np, int rows, float c, Release release) {
   float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
   if (np == 0) release();
@@ -57,14 +64,14 @@ __device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, 
         tmem_ld16(taddr + ch * 16 + 16, v + 16);
         tmem_ld_wait_for(v);
         if (k + 2 >= np) release();
-        colsum_piece<kFull>(v, lse_s + ch * 16, valid, c, acc, acc1);
-        colsum_piece<kFull>(v + 16, lse_s + ch * 16 + 16, valid - 16, c, acc, acc1);
+        colsum_piece<kFull, kFold>(v, lse_s + ch * 16, valid, c, acc, acc1);
+        colsum_piece<kFull, kFold>(v + 16, lse_s + ch * 16 + 16, valid - 16, c, acc, acc1);
       } else {
         uint32_t v[16];
         tmem_ld16(taddr + ch * 16, v);
         tmem_ld_wait_for16(v);
         release();
-        colsum_piece<kFull>(v, lse_s + ch * 16, valid, c, acc, acc1);
+        colsum_piece<kFull, kFold>(v, lse_s + ch * 16, valid, c, acc, acc1);
       }
     }
   }
@@ -73,7 +80,7 @@ __device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, 
 
 // The same with 16-column loads one piece ahead: the tensor-memory load of piece k + 1 is in flight while
 // piece k's exponentials run.
-template <bool kFull, class Release>
+template <bool kFull, bool kFold, class Release>
 __device__ __forceinline__ float colsum_job_ahead(uint32_t taddr, const float* lse_s, int p0, int np, int rows, float c, Release release) {
   float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
   if (np == 0) {
@@ -90,7 +97,7 @@ __device__ __forceinline__ float colsum_job_ahead(uint32_t taddr, const float* l
       uint32_t* nxt = (k & 1) ? va : vb;
       if (k + 1 < np) tmem_ld16(taddr + (p0 + k + 1) * 16, nxt);
       else release();
-      colsum_piece<kFull>(cur, lse_s + (p0 + k) * 16, rows - (p0 + k) * 16, c, acc, acc1);
+      colsum_piece<kFull, kFold>(cur, lse_s + (p0 + k) * 16, rows - (p0 + k) * 16, c, acc, acc1);
       if (k + 1 < np) tmem_ld_wait_for16(nxt);
     }
   }
@@ -114,6 +121,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   using T = TileGeo<kTile2>;
+  constexpr bool kFold = kConvert;                              // the library's own fp16 queries arrive scaled: -lse rides on the MMAs
   const int kvh = blockIdx.y;
   const Work w = cta_work(t, ct, a, kTile2, false);
   const int nt = w.nt, L = w.L, b = w.b;
@@ -135,8 +143,10 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // ============================================================================= MMA issuer
     if (lane == 0) {
       bool ok = wt.wait(bars.q_full(), 0);
+      if (ok && kFold) ok = wt.wait(bars.lse_ready(), 0);
       const uint32_t idesc = kConvert ? umma_idesc_f16(128, ncols) : umma_idesc(128, ncols);
       const uint64_t qd = umma_desc(sbase);
+      const uint64_t ones_d = umma_desc_rows32(sbase + kOnesSlab), lse_d = umma_desc_rows32(sbase + kLseSlab);
       const uint32_t ring = sbase + 2 * q_half;
       Ring rs(S), ra(n_acc);
       for (int ti = 0; ti < nt && ok; ++ti, rs.next(), ra.next()) {
@@ -152,6 +162,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
           const int half = ks >> 2, kk = ks & 3;
           umma_ss(d, desc_advance(kd, half * T::kHalf + kk * 32), desc_advance(qd, half * q_half + kk * 32), idesc, ks ? 1u : 0u);
         }
+        if (kFold) umma_ss(d, ones_d, lse_d, idesc, 1u);        // D[key, i] += 1 * (-lse_i) (an fp16 pair against two ones)
         tc_commit(bars.acc_full(buf));
         tc_commit(bars.k_empty(s));                             // the K stage is free once these MMAs retire
       }
@@ -213,8 +224,25 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
           if (a.lse_out && w.chunk == ct.cu_chunk[b]) a.lse_out[w.qrow_base + grow] = l2 * 0.6931471805599453f;
         }
         lse_s[row] = -l2;                                       // negated: the epilogue adds it
+        if (kFold) {
+          // row `row` of the [256 x 16] operand: (-lse) as an fp16 pair in channels 0 and 1, zeros elsewhere.
+          // The ones operand carries its two ones in BOTH 16-byte halves of every row, so whichever way the
+          // 32-byte swizzle orders the halves of a row, the k-step adds exactly hi + lo.
+          const __half hi = __float2half_rn(-l2);
+          const __half lo = __float2half_rn(live ? -l2 - __half2float(hi) : 0.f);
+          const uint32_t pair = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+          const uint32_t dst = sbase + kLseSlab + (row >> 3) * 256 + (row & 7) * 32;
+          sts128(dst, make_uint4(live ? pair : 0u, 0u, 0u, 0u));
+          sts128(dst + 16, make_uint4(0u, 0u, 0u, 0u));
+        }
+      }
+      if (kFold) {
+        const int tid_e = (warp - kFirstEpiWarp) * 32 + lane;   // 0 .. 511: the ones operand, 256 pieces of 16 bytes
+        if (tid_e < kOnesSlabBytes / 16) sts128(sbase + kOnesSlab + tid_e * 16, make_uint4(0x3c003c00u, 0u, 0u, 0u));
+        fence_proxy_async();                                    // the MMAs read both operands through the async proxy
       }
       epilogue_sync();
+      if (kFold && warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());
     }
     // Pieces of a job (16 query columns): group g takes pieces [g nch / 4, (g + 1) nch / 4), at most four
     const int nch = ncols >> 4;
@@ -234,9 +262,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.acc_empty(buf));
       };
-      const float sum = !full             ? colsum_job<false>(taddr, lse_s, p0, np, w.rows, c, release)
-                        : DAPQ_TMEM_AHEAD ? colsum_job_ahead<true>(taddr, lse_s, p0, np, w.rows, c, release)
-                                          : colsum_job<true>(taddr, lse_s, p0, np, w.rows, c, release);
+      const float sum = !full             ? colsum_job<false, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
+                        : DAPQ_TMEM_AHEAD ? colsum_job_ahead<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
+                                          : colsum_job<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release);
       const int slot = ti % kExchDepth;
       if (ti >= kExchDepth) ok = __all_sync(0xffffffffu, wt.wait(bars.part_empty(slot), ((ti / kExchDepth) - 1) & 1));
       if (!ok) break;

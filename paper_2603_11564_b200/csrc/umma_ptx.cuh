@@ -109,6 +109,12 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
   return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
          (2ull << 61);
 }
+// The same for a K-major operand whose rows are 32 bytes (16 half-precision channels, one MMA k-step) with
+// the 32-byte swizzle: 8-row groups 256 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_rows32(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(256 >> 4) << 32) | (1ull << 46) |
+         (6ull << 61);
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, shape M x N.
 __host__ __device__ constexpr uint32_t umma_idesc(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
