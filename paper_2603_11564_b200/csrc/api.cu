@@ -212,7 +212,7 @@ bool wants_umma(const dapq_ctx* ctx) {
 dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& t, const float* lse_in,
                            float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
   cudaError_t e = launch_score_umma(plan, t, ctx->dims, lse_in, ctx->part, scores, score_stride,
-                                    lse_out, ctx->status, s, &ctx->log);
+                                    lse_out, ctx->status, ctx->wait_limit, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels (two-part bf16 queries)");
   return DAPQ_OK;
 }

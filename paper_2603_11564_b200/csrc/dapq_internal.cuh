@@ -154,7 +154,7 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
 int64_t umma_part_elems(int max_batch, int n_q_heads, int n_kv_heads, int n_pseudo);
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
                               float2* part, float* scores, int64_t score_stride, float* lse_out,
-                              int* status, cudaStream_t s, LaunchLog* log);
+                              int* status, long long wait_limit, cudaStream_t s, LaunchLog* log);
 
 // Pieces shared by the two tensor-core scorers (defined in score_qg.cu): the TMA descriptor of a
 // 16-bit [.., rows, 128] tensor (boxes of 64 channels x box_rows rows, 128-byte swizzle), and the cut of

@@ -102,7 +102,7 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
-      int li = 0;
+      int li = 0, n_done = 0;
       uint32_t use0 = 0u, use1 = 0u;                            // jobs issued into each accumulator
       bool ok = true;
       const uint32_t idesc = umma_idesc(128, kTile1);
@@ -110,17 +110,17 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
         const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
         const int mb = (rows_g + 127) / 128;
-        ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
+        ok = mbar_wait_limit(bars.q_full(), qg & 1, abort_flag, a.status, a.wait_limit);
         for (int ti = 0; ti < nt && ok; ++ti, ++li) {
           const int s = li % kStages1;
-          ok = mbar_wait(bars.k_full(s), (li / kStages1) & 1, abort_flag, a.status);
+          ok = mbar_wait_limit(bars.k_full(s), (li / kStages1) & 1, abort_flag, a.status, a.wait_limit);
           if (!ok) break;
           const uint64_t kd = umma_desc(sbase + G::k + s * kStageBytes1);
           for (int m = 0; m < mb && ok; ++m) {
             // two blocks: block m -> accumulator m; one block: tiles alternate between the two
             const int buf = (mb == 2) ? m : (ti & 1);
             const uint32_t used = buf ? use1 : use0;
-            if (used) ok = mbar_wait(bars.acc_empty(buf), (used - 1) & 1, abort_flag, a.status);
+            if (used) ok = mbar_wait_limit(bars.acc_empty(buf), (used - 1) & 1, abort_flag, a.status, a.wait_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d = tmem_base + buf * kTile1;
@@ -145,7 +145,9 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           tc_commit(bars.k_empty(s));                           // the K stage is free once these MMAs retire
         }
         tc_commit(bars.q_empty());
+        ++n_done;
       }
+      mma_drain(bars, n_done, n_done < a.n_qgroups);
     }
   } else {
     // ============================================================================== epilogue
@@ -171,7 +173,7 @@ score_sweep1_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         for (int m = 0; m < mb && ok; ++m) {
           const int buf = (mb == 2) ? m : (ti & 1);
           const uint32_t used = buf ? use1 : use0;
-          ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), used & 1, abort_flag, a.status));
+          ok = __all_sync(0xffffffffu, mbar_wait_limit(bars.acc_full(buf), used & 1, abort_flag, a.status, a.wait_limit));
           if (!ok) break;
           if (buf) ++use1; else ++use0;
           tc_fence_after();

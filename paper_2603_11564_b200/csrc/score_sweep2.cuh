@@ -51,17 +51,17 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
-      int job = 0;                                              // = K tiles consumed: one job per tile
+      int job = 0, n_done = 0;                                  // job = K tiles consumed: one job per tile
       bool ok = true;
       const uint64_t qd_hi = umma_desc(sbase + G::q_hi), qd_lo = umma_desc(sbase + G::q_lo);
       for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
         const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
         const uint32_t idesc = umma_idesc(128, kWide ? 256 : (rows_g + 15) & ~15);   // only the query columns that exist
-        ok = mbar_wait(bars.q_full(), qg & 1, abort_flag, a.status);
+        ok = mbar_wait_limit(bars.q_full(), qg & 1, abort_flag, a.status, a.wait_limit);
         for (int ti = 0; ti < nt && ok; ++ti, ++job) {
           const int s = job % kStages2, buf = job % kAcc;
-          ok = mbar_wait(bars.k_full(s), (job / kStages2) & 1, abort_flag, a.status);
-          if (ok && job >= kAcc) ok = mbar_wait(bars.acc_empty(buf), ((job / kAcc) - 1) & 1, abort_flag, a.status);
+          ok = mbar_wait_limit(bars.k_full(s), (job / kStages2) & 1, abort_flag, a.status, a.wait_limit);
+          if (ok && job >= kAcc) ok = mbar_wait_limit(bars.acc_empty(buf), ((job / kAcc) - 1) & 1, abort_flag, a.status, a.wait_limit);
           if (!ok) break;
           tc_fence_after();
           const uint64_t kd = umma_desc(sbase + G::k + s * kStageBytes2);
@@ -94,7 +94,9 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           tc_commit(bars.k_empty(s));                           // the K stage is free once these MMAs retire
         }
         tc_commit(bars.q_empty());
+        ++n_done;
       }
+      mma_drain(bars, n_done, n_done < a.n_qgroups);
     }
   } else {
     // ============================================================================== epilogue
@@ -167,7 +169,7 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
       for (int ti = 0; ti < nt && ok; ++ti, ++job) {
         const int buf = job % kAcc;
-        ok = __all_sync(0xffffffffu, mbar_wait(bars.acc_full(buf), (job / kAcc) & 1, abort_flag, a.status));
+        ok = __all_sync(0xffffffffu, mbar_wait_limit(bars.acc_full(buf), (job / kAcc) & 1, abort_flag, a.status, a.wait_limit));
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = lane_addr + buf * kAccCols;
@@ -239,13 +241,13 @@ score_sweep2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         // written once group 0 has read the job before (part_empty) and read once all three have
         // written (part_full).
         if (eg > 0) {
-          if (job > 0) ok = __all_sync(0xffffffffu, mbar_wait(bars.part_empty(), (job - 1) & 1, abort_flag, a.status));
+          if (job > 0) ok = __all_sync(0xffffffffu, mbar_wait_limit(bars.part_empty(), (job - 1) & 1, abort_flag, a.status, a.wait_limit));
           if (!ok) break;
           exch[(eg - 1) * 128 + r] = sum;
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.part_full());         // (release: the stores above are visible to the waiter)
         } else {
-          ok = __all_sync(0xffffffffu, mbar_wait(bars.part_full(), job & 1, abort_flag, a.status));
+          ok = __all_sync(0xffffffffu, mbar_wait_limit(bars.part_full(), job & 1, abort_flag, a.status, a.wait_limit));
           if (!ok) break;
           sum += (exch[r] + exch[128 + r]) + exch[256 + r];
           __syncwarp();

@@ -73,7 +73,7 @@ bool umma_plan(const void* q_hi, int has_lo, int64_t lo_row_offset, const CacheD
 
 cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in,
                               float2* part, float* scores, int64_t score_stride, float* lse_out,
-                              int* status, cudaStream_t s, LaunchLog* log) {
+                              int* status, long long wait_limit, cudaStream_t s, LaunchLog* log) {
   UmmaArgs a;
   a.n_pseudo = dm.n_pseudo;
   a.group = dm.group;
@@ -87,6 +87,7 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
   a.has_lo = plan.has_lo;
   a.lo_row_offset = (int32_t)plan.lo_row_offset;
   a.scale_log2e = dm.scale_log2e;
+  a.wait_limit = wait_limit > 0 ? wait_limit : ptx::kWaitLimit;
   a.part = part;
   a.lse_in = lse_in;
   a.lse_out = lse_out;

@@ -65,6 +65,7 @@ struct UmmaArgs {
   int32_t has_lo;            // the query operand carries a low-order bf16 part
   int32_t lo_row_offset;     // rows between the hi and the lo copy in the query tensor
   float scale_log2e;
+  long long wait_limit;      // cycles a wait may take before the CTA gives up
   float2* part;              // [n_chunks1, H_kv, rows_pad] (running max, sum) of every query row over a chunk's keys, base 2
   const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
   float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
@@ -153,7 +154,7 @@ template <class G, int kTile, int kStages, int kStage, int kHalf, bool kSideBySi
 __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w,
                                              const UmmaArgs& a, uint32_t sbase, const Bars& bars, int kvh,
                                              volatile int* abort_flag) {
-  int li = 0;                                               // K tiles loaded so far
+  int li = 0, n_q = 0;                                      // K tiles / query groups loaded so far
   bool ok = true;
   auto load_tile = [&](int ti) {
     const int s = li % kStages;
@@ -171,10 +172,11 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
   for (int qg = 0; qg < a.n_qgroups && ok; ++qg) {
     const int rows_g = min(G::kRows, a.rows_total - qg * G::kRows);
     const int mb = (rows_g + 127) / 128;
-    if (qg > 0) ok = mbar_wait(bars.q_empty(), (qg - 1) & 1, abort_flag, a.status);
+    if (qg > 0) ok = mbar_wait_limit(bars.q_empty(), (qg - 1) & 1, abort_flag, a.status, a.wait_limit);
     if (!ok) break;
     const int parts = a.has_lo ? 2 : 1;
     mbar_expect_tx(bars.q_full(), (uint32_t)(parts * mb * 2 * 128 * 128));
+    ++n_q;
     for (int part = 0; part < parts; ++part)
       for (int half = 0; half < 2; ++half)
         for (int m = 0; m < mb; ++m)
@@ -183,19 +185,28 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
                       tm_q, bars.q_full(), half * 64, part * a.lo_row_offset + w.qrow_base + qg * G::kRows + m * 128);
     for (int ti = (qg == 0 ? n_first : 0); ti < w.nt; ++ti) {
       const int s = li % kStages;
-      if (li >= kStages) ok = mbar_wait(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status);
+      if (li >= kStages) ok = mbar_wait_limit(bars.k_empty(s), ((li / kStages) - 1) & 1, abort_flag, a.status, a.wait_limit);
       if (!ok) break;
       load_tile(ti);
     }
   }
-  if (!ok) {
-    // aborting: let the copies already issued land before the CTA returns
-    for (int back = 1; back <= kStages && back <= li; ++back) {
-      const int l2 = li - back;
-      const long long start = clock64();
-      while (!mbar_try(bars.k_full(l2 % kStages), (l2 / kStages) & 1) && clock64() - start < kWaitLimit) {}
-    }
+  // See every copy issued above land before this thread (and with it the CTA) returns: in a normal run they
+  // have all been consumed by now; in an aborting CTA nobody else may be left to wait for them.
+  for (int back = 1; back <= kStages && back <= li; ++back) {
+    const int l2 = li - back;
+    drain_wait(bars.k_full(l2 % kStages), (l2 / kStages) & 1, kWaitLimit);
   }
+  if (n_q > 0) drain_wait(bars.q_full(), (n_q - 1) & 1, kWaitLimit);
+}
+
+// The MMA issuer's last act: see every MMA it issued retire before tensor memory is given back.  q_empty
+// receives one commit per finished query group (n_done so far); an issuer that left its loop early adds one.
+__device__ __forceinline__ void mma_drain(const Bars& bars, int n_done, bool left_early) {
+  if (left_early) {
+    tc_commit(bars.q_empty());
+    ++n_done;
+  }
+  if (n_done > 0) drain_wait(bars.q_empty(), (n_done - 1) & 1, kWaitLimit);
 }
 
 }  // namespace umma

@@ -60,7 +60,11 @@ __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, v
       atomicOr(status, kStatusTimeout);
       return false;
     }
-    if (mbar_try_suspend(bar, parity, 20000u)) return true;
+    // (a burst of suspended tries between two looks at the flag and the clock: a waiting warp should cost the
+    // schedulers as few instructions as possible, they are the epilogue's)
+#pragma unroll 1
+    for (int it = 0; it < 16; ++it)
+      if (mbar_try_suspend(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
   }
 }

@@ -730,14 +730,16 @@ def test_evict_layers_full_size_sampled_heads(dq):
 
 
 # ------------------------------------------------------------------ a device-side wait that runs out
-def test_wait_limit_gives_up_reports_timeout_and_recovers(dq):
+@pytest.mark.parametrize("flags", [0, 8 | 16])
+def test_wait_limit_gives_up_reports_timeout_and_recovers(dq, flags):
     """With the wait bound set to one cycle, the first wait of every score CTA that is not satisfied at once
     runs out: the kernels return normally, dapq_poll_status reports DAPQ_ERR_TIMEOUT once and clears the
-    status word, and the same context then computes the right answer again."""
+    status word, and the same context then computes the right answer again.  Both tensor-core scorers (flags 0:
+    fp16 queries; 8 | 16: the older kernels with the two-part bf16 operand)."""
     w = gi.scaled_down("llama3_8b_32k", 8, n_layers=1)
     data = util.make_case(w)
     ref = util.oracle_evict(w, data)
-    ctx = _ctx(dq, w)
+    ctx = _ctx(dq, w, flags=flags)
     good = _gpu_evict(dq, w, data, ctx)
     dq.dapq_set_wait_limit(ctx, 1)
     q, k, v = (data[x].cuda() for x in ("q_pre", "k", "v"))
