@@ -57,10 +57,24 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Sum of the query groups' score slots, in slot order (one thread per score).
+// Sum of the query groups' score slots, in slot order (one thread per four scores; n4 = count / 4).
 __global__ void __launch_bounds__(256)
-score_slots_sum_kernel(const float* __restrict__ slots, int n_slots, int64_t slot_stride, float* __restrict__ scores,
-                       int64_t count) {
+score_slots_sum_kernel(const float4* __restrict__ slots, int n_slots, int64_t slot_stride4, float4* __restrict__ scores,
+                       int64_t n4) {
+  pdl_wait();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n4) return;
+  float4 v = slots[i];
+  for (int s = 1; s < n_slots; ++s) {
+    const float4 u = slots[s * slot_stride4 + i];
+    v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+  }
+  scores[i] = v;
+}
+// The same one score per thread (arrays whose length or address is no multiple of 16 bytes).
+__global__ void __launch_bounds__(256)
+score_slots_sum1_kernel(const float* __restrict__ slots, int n_slots, int64_t slot_stride, float* __restrict__ scores,
+                        int64_t count) {
   pdl_wait();
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= count) return;
@@ -194,8 +208,12 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
   if (plan.n_qgroups > 1) {
     const int64_t count = (int64_t)dm.n_kv_heads * score_stride;
     log->begin(kKindSlotSum, s);
-    e = launch_pdl(score_slots_sum_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, s, 1, (const float*)slots,
-                   plan.n_qgroups, a.slot_stride, scores, count);
+    if (count % 4 == 0 && a.slot_stride % 4 == 0 && ((uintptr_t)slots & 15u) == 0 && ((uintptr_t)scores & 15u) == 0)
+      e = launch_pdl(score_slots_sum_kernel, dim3((unsigned)((count / 4 + 255) / 256)), dim3(256), 0, s, 1,
+                     (const float4*)slots, plan.n_qgroups, a.slot_stride / 4, (float4*)scores, count / 4);
+    else
+      e = launch_pdl(score_slots_sum1_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, s, 1, (const float*)slots,
+                     plan.n_qgroups, a.slot_stride, scores, count);
     log->end(s);
     if (e != cudaSuccess) return e;
   }

@@ -14,23 +14,13 @@ constexpr int kTile1 = 192;                    // keys per K tile of sweep 1 (= 
 constexpr int kTile2 = 128;                    // keys per K tile of sweep 2 (= UMMA M there)
 constexpr int kGroupRows = 256;                // most query rows a CTA keeps resident
 constexpr int kEpiGroups = 4;                  // epilogue groups of 4 warps (128 TMEM lanes each)
-#ifndef DAPQ_CONV_WARPS
-#define DAPQ_CONV_WARPS 4
-#endif
-constexpr int kConvWarps = DAPQ_CONV_WARPS;    // warps that convert the K tiles in place
+constexpr int kConvWarps = 4;                  // warps that convert the K tiles in place
 constexpr int kFirstEpiWarp = 2 + kConvWarps;
 constexpr int kEpiThreads = kEpiGroups * 128;
 constexpr int kThreads1 = (kFirstEpiWarp + 4 * kEpiGroups) * 32;        // sweep 1: 22 warps
 constexpr int kThreads2 = kThreads1 + 32;                               // sweep 2: one more warp sums the groups' partials
 constexpr int kTmemCols = 512;
-#ifndef DAPQ_MAX_STAGES
-#define DAPQ_MAX_STAGES 4
-#endif
-#ifndef DAPQ_L2_AHEAD
-#define DAPQ_L2_AHEAD 0
-#endif
-constexpr int kMaxStages = DAPQ_MAX_STAGES, kMaxAcc = 4;
-constexpr int kL2Ahead = DAPQ_L2_AHEAD;        // tiles beyond the ring that the producer asks L2 for (0: none)
+constexpr int kMaxStages = 4, kMaxAcc = 4;
 constexpr int kExchDepth = 4;                  // jobs whose partial sums can wait in shared memory (sweep 2)
 constexpr int kRingEnd = 216 * 1024;           // queries + K ring end here; the small state follows
 // Sweep 2 with its own fp16 queries appends one k-step to every job's MMAs that adds -lse_i to column i of
@@ -204,10 +194,6 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     const int row = w.row_base + (w.t0 + ti) * kTile;
     tma_load_3d(ring + s * T::kStage, tm_k, bars.k_full(s), 0, row, kvh);
     tma_load_3d(ring + s * T::kStage + T::kHalf, tm_k, bars.k_full(s), 64, row, kvh);
-    if (kL2Ahead > 0 && ti + kL2Ahead < w.nt) {
-      tma_prefetch_3d(tm_k, 0, row + kL2Ahead * kTile, kvh);
-      tma_prefetch_3d(tm_k, 64, row + kL2Ahead * kTile, kvh);
-    }
     ++li;
   };
   load_tile(0);                                             // (w.nt >= 1: checked by the caller)

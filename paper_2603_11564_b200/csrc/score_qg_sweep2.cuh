@@ -78,36 +78,6 @@ __device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, 
   return (acc.x + acc.y) + (acc1.x + acc1.y);
 }
 
-// The same with 16-column loads one piece ahead: the tensor-memory load of piece k + 1 is in flight while
-// piece k's exponentials run.
-template <bool kFull, bool kFold, class Release>
-__device__ __forceinline__ float colsum_job_ahead(uint32_t taddr, const float* lse_s, int p0, int np, int rows, float c, Release release) {
-  float2 acc = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-  if (np == 0) {
-    release();
-    return 0.f;
-  }
-  uint32_t va[16], vb[16];
-  tmem_ld16(taddr + p0 * 16, va);
-  tmem_ld_wait_for16(va);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    if (k < np) {
-      uint32_t* cur = (k & 1) ? vb : va;
-      uint32_t* nxt = (k & 1) ? va : vb;
-      if (k + 1 < np) tmem_ld16(taddr + (p0 + k + 1) * 16, nxt);
-      else release();
-      colsum_piece<kFull, kFold>(cur, lse_s + (p0 + k) * 16, rows - (p0 + k) * 16, c, acc, acc1);
-      if (k + 1 < np) tmem_ld_wait_for16(nxt);
-    }
-  }
-  return (acc.x + acc.y) + (acc1.x + acc1.y);
-}
-
-#ifndef DAPQ_TMEM_AHEAD
-#define DAPQ_TMEM_AHEAD 0
-#endif
-
 template <bool kConvert>
 __global__ void __launch_bounds__(kThreads2, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
@@ -262,9 +232,8 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.acc_empty(buf));
       };
-      const float sum = !full             ? colsum_job<false, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
-                        : DAPQ_TMEM_AHEAD ? colsum_job_ahead<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
-                                          : colsum_job<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release);
+      const float sum = full ? colsum_job<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
+                             : colsum_job<false, kFold>(taddr, lse_s, p0, np, w.rows, c, release);
       const int slot = ti % kExchDepth;
       if (ti >= kExchDepth) ok = __all_sync(0xffffffffu, wt.wait(bars.part_empty(slot), ((ti / kExchDepth) - 1) & 1));
       if (!ok) break;
