@@ -220,7 +220,7 @@ dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& 
 dapq_status run_score_qg(dapq_ctx* ctx, const QgPlan& plan, const SeqTable& t, const float* lse_in,
                          float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
   cudaError_t e = launch_score_qg(plan, t, ctx->dims, lse_in, ctx->part, ctx->slots, scores, score_stride, lse_out,
-                                  ctx->status, ctx->wait_limit, s, &ctx->log);
+                                  ctx->lse2, ctx->status, ctx->wait_limit, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels");
   return DAPQ_OK;
 }
@@ -552,8 +552,11 @@ dapq_status evict_impl(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
   if (wants_umma(ctx) && !wants_lo(ctx) && qg_plan(ctx->q_rot, (flags & DAPQ_FLAG_Q_BF16) ? 0 : 1, cd, t, ctx->dims, ctx->n_sm, &qplan)) {
     // tensor-core scorer: rotated queries rounded to fp16, K tiles converted to fp16 on their way to the MMAs
     // (DAPQ_FLAG_Q_BF16: queries rounded to bf16, no conversion)
+    // (with fp16 queries the rotation also leaves, in lse2, every query's logit against the first key of its
+    // sequence: the reference that sweep 1 measures the row's other logits against)
+    const RopeRef ref = {(const __nv_bfloat16*)cd.k, cd.k_head_stride, cd.k_row_stride, ctx->lse2, ctx->dims.group};
     e = launch_rope(ctx->shape.dtype, qplan.q_is_f16 ? kRopeOutF16 : kRopeOutBf16, 0, q_pre, ctx->q_rot, ctx->inv_freq, t,
-                    ctx->dims, after_own_compaction, s, &ctx->log);
+                    ctx->dims, after_own_compaction, s, &ctx->log, &ref);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
     st = run_score_qg(ctx, qplan, t, nullptr, scores, score_stride, nullptr, s);
   } else if (wants_umma(ctx) && wants_lo(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {

@@ -122,8 +122,17 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 // q_pre has element type `dtype`; q_rot is written as `out_mode`: bf16, fp32 (unrounded, for
 // the CUDA-core scorer) or a bf16 pair hi + lo with lo = bf16(q - hi) stored `lo_offset`
 // elements after hi (for the tensor-core scorer).
+// ref (fp16 output mode only, may be NULL): the bf16 key cache and where to write, per rotated query, its base-2
+// logit against the first key of its sequence (see rope.cu).
+struct RopeRef {
+  const __nv_bfloat16* k;
+  int64_t head_stride, row_stride;   // elements
+  float* out;                        // [B, H_q, N]
+  int32_t group;
+};
 cudaError_t launch_rope(int dtype, int out_mode, int64_t lo_offset, const void* q_pre, void* q_rot, const double* inv_freq_dev,
-                        const SeqTable& t, const Dims& dm, bool late_wait, cudaStream_t s, LaunchLog* log);
+                        const SeqTable& t, const Dims& dm, bool late_wait, cudaStream_t s, LaunchLog* log,
+                        const RopeRef* ref = nullptr);
 
 // Generic CUDA-core scorer (any N <= 128, both dtypes).
 //   part  : [n_chunks, H_q, N] float2 (running max, sum) in base-2 logits, room for max_chunks
@@ -174,8 +183,9 @@ struct QgPlan {
 };
 int qg_groups(const Dims& dm);
 bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t, const Dims& dm, int n_sm, QgPlan* plan);
+// ref: with fp16 queries, the [B, H_q, N] reference logits that the rotation kernel wrote beside them.
 cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in, float2* part,
-                            float* slots, float* scores, int64_t score_stride, float* lse_out, int* status,
+                            float* slots, float* scores, int64_t score_stride, float* lse_out, const float* ref, int* status,
                             long long wait_limit, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,

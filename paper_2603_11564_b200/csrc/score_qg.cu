@@ -142,7 +142,7 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
   plan->rows_g = (((rows_total + plan->n_qgroups - 1) / plan->n_qgroups) + 15) & ~15;
   plan->q_is_f16 = q_is_f16;
   const int q_bytes = ((plan->rows_g + 127) / 128) * 2 * 128 * 128;
-  const int s1 = (kRingEnd - q_bytes) / TileGeo<kTile1>::kStage;
+  const int s1 = (kRingEnd - (q_is_f16 ? kRefSlabBytes : 0) - q_bytes) / TileGeo<kTile1>::kStage;   // (the reference operand sits at the end)
   const int s2 = (kRingEnd - (q_is_f16 ? kSlabBytes : 0) - q_bytes) / TileGeo<kTile2>::kStage;   // (the -lse operands sit at the end)
   plan->n_stages1 = s1 < kMaxStages ? s1 : kMaxStages;
   plan->n_stages2 = s2 < kMaxStages ? s2 : kMaxStages;
@@ -163,7 +163,7 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
 }
 
 cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in, float2* part,
-                            float* slots, float* scores, int64_t score_stride, float* lse_out, int* status,
+                            float* slots, float* scores, int64_t score_stride, float* lse_out, const float* ref, int* status,
                             long long wait_limit, cudaStream_t s, LaunchLog* log) {
   Args a;
   a.n_pseudo = dm.n_pseudo;
@@ -177,6 +177,7 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
   a.scale_log2e = plan.q_is_f16 ? 1.f : dm.scale_log2e;        // the library's own fp16 queries are stored times scale * log2(e)
   a.wait_limit = wait_limit > 0 ? wait_limit : kWaitLimit;
   a.part = part;
+  a.ref = ref;
   a.lse_in = lse_in;
   a.lse_out = lse_out;
   a.score_stride = score_stride;

@@ -28,6 +28,9 @@ constexpr int kRingEnd = 216 * 1024;           // queries + K ring end here; the
 constexpr int kLseSlabBytes = kGroupRows * 32, kOnesSlabBytes = kTile2 * 32;
 constexpr int kSlabBytes = kLseSlabBytes + kOnesSlabBytes;                      // kept at the end of the ring area
 constexpr int kLseSlab = kRingEnd - kSlabBytes, kOnesSlab = kRingEnd - kOnesSlabBytes;
+// Sweep 1 does the same with a per-row reference logit (its [256 x 16] operand also sits at the end of the
+// ring area; its [192 x 16] operand of ones takes the place of sweep 2's exchange ring behind the barriers).
+constexpr int kRefSlabBytes = kGroupRows * 32, kRefSlab = kRingEnd - kRefSlabBytes, kOnes1SlabBytes = kTile1 * 32;
 
 template <int kTile>
 struct TileGeo {
@@ -48,7 +51,8 @@ struct Smem {
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
-static_assert(Smem::lse % 16 == 0 && Smem::aux % 16 == 0 && Smem::exch % 16 == 0, "vector loads need 16-byte alignment");
+static_assert(Smem::lse % 16 == 0 && Smem::aux % 16 == 0 && Smem::exch % 256 == 0, "vector loads need 16-byte alignment, MMA operands 256");
+static_assert(kOnes1SlabBytes <= kExchDepth * kEpiGroups * 128 * 4, "sweep 1's operand of ones does not fit the exchange area");
 constexpr int kSmemBytes = Smem::total;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
@@ -62,6 +66,7 @@ struct Args {
   float scale_log2e;
   long long wait_limit;      // cycles a wait may take before the CTA gives up
   float2* part;              // [n_chunks1, H_kv, rows_pad] (running max, sum) of every query row over a chunk's keys, base 2
+  const float* ref;          // [B, H_q, N] base-2 reference logit of every query row (fp16 queries only)
   const float* lse_in;       // [B, H_q, N] natural-log lse from the caller, or NULL (use part)
   float* lse_out;            // [B, H_q, N] natural-log lse used, or NULL
   float* scores;             // [n_qgroups][H_kv][score_stride] when n_qgroups > 1 (one slot per group), else [H_kv][score_stride]

@@ -73,6 +73,56 @@ __device__ __forceinline__ float2 merge_stats(float2 a, float2 b) {
   return make_float2(m, a.y * exp2f(a.x - m) + b.y * exp2f(b.x - m));
 }
 
+// Row statistics without a running maximum.  With the library's own fp16 queries every job's MMAs end with
+// one more k-step that subtracts a per-row reference logit r (the row's logit against the first key of its
+// sequence, written by the rotation kernel), so the accumulator holds x = logit - r and a job is just
+// z += sum 2^x: no maximum, no rescaling, no subtraction.  The sum of a row is kept as z * 2^m with m = r
+// at first.  The result stays exact for every input: a job whose sum leaves the float range (a key more
+// than ~2^127 above the reference) is redone from its registers with its own maximum and merged, which
+// moves m; once m is far from r every job takes that careful path.  Logits far BELOW r only underflow
+// against a term, the reference key's own, that is part of the same row's total.
+struct RowSum {
+  float r, m, z, sc;                                            // reference, base of z, sum, 2^(r - m)
+  __device__ __forceinline__ void init(float ref) { r = m = ref; z = 0.f; sc = 1.f; }
+};
+template <bool kMasked>
+__device__ __forceinline__ void row_sum_cols(uint32_t* v, int col0, int lim, RowSum& st) {
+  float* x = reinterpret_cast<float*>(v);
+  if (kMasked) {
+#pragma unroll
+    for (int e = 0; e < kCols1; ++e)
+      if (col0 + e > lim) x[e] = -CUDART_INF_F;
+  }
+  if (st.m - st.r < 100.f) {
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int e = 0; e < kCols1; e += 4) {
+      const float2 x0 = make_float2(x[e], x[e + 1]), x1 = make_float2(x[e + 2], x[e + 3]);
+      acc0 = __fadd2_rn(acc0, ((kPolyPairMask >> ((e / 2) & 15)) & 1u) ? ex2_pair_poly<true>(x0) : ex2_pair_mufu(x0));
+      acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> ((e / 2 + 1) & 15)) & 1u) ? ex2_pair_poly<true>(x1) : ex2_pair_mufu(x1));
+    }
+    const float zj = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+    if (zj < 1e37f) {                                           // (false for inf and NaN too)
+      st.z = fmaf(zj, st.sc, st.z);
+      if (st.z > 1e30f) {                                       // keep z well inside the float range
+        st.m += 64.f;
+        st.z *= 5.421010862427522e-20f;                         // 2^-64
+        st.sc *= 5.421010862427522e-20f;
+      }
+      return;
+    }
+  }
+  // careful path: this job's own maximum and sum (relative to r), merged into the row's
+  float ml = -CUDART_INF_F, zl = 0.f;
+  row_stats_cols<kMasked>(v, col0, lim, 1.f, ml, zl);
+  if (ml > -CUDART_INF_F) {
+    const float2 mg = merge_stats(make_float2(st.m, st.z), make_float2(st.r + ml, zl));
+    st.m = mg.x;
+    st.z = mg.y;
+    st.sc = exp2f(st.r - st.m);
+  }
+}
+
 template <bool kConvert>
 __global__ void __launch_bounds__(kThreads1, 1)
 rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
@@ -85,6 +135,7 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   using T = TileGeo<kTile1>;
+  constexpr bool kFold = kConvert;                              // the library's own fp16 queries come with reference logits
   const int kvh = blockIdx.y;
   const Work w = cta_work(t, ct, a, kTile1, true);
   const int nt = w.nt, L = w.L, N = a.n_pseudo, mb = w.mb;
@@ -102,8 +153,10 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (lane == 0) {
       uint32_t use0 = 0u, use1 = 0u;                            // jobs issued into each accumulator
       bool ok = wt.wait(bars.q_full(), 0);
+      if (ok && kFold) ok = wt.wait(bars.lse_ready(), 0);
       const uint32_t idesc = kConvert ? umma_idesc_f16(128, kTile1) : umma_idesc(128, kTile1);
       const uint64_t qd = umma_desc(sbase);
+      const uint64_t ref_d = umma_desc_rows32(sbase + kRefSlab), ones_d = umma_desc_rows32(sbase + Smem::exch);
       const uint32_t ring = sbase + 2 * q_half;
       Ring rs(S);
       for (int ti = 0; ti < nt && ok; ++ti, rs.next()) {
@@ -125,6 +178,7 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const int half = ks >> 2, kk = ks & 3;
             umma_ss(d, desc_advance(qm, half * q_half + kk * 32), desc_advance(kd, half * T::kHalf + kk * 32), idesc, ks ? 1u : 0u);
           }
+          if (kFold) umma_ss(d, desc_advance(ref_d, m * 128 * 32), ones_d, idesc, 1u);   // D[i, key] += (-r_i) * 1
           tc_commit(bars.acc_full(buf));
           if (buf) ++use1; else ++use0;
         }
@@ -147,7 +201,36 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     bool ok = true;
     // running max (raw dot product) and sum of this thread's row of block 0 / block 1
     float m_raw0 = -CUDART_INF_F, z0 = 0.f, m_raw1 = -CUDART_INF_F, z1 = 0.f;
+    RowSum rs0, rs1;                                            // ... or, with reference logits, the rows' sums
     const int i_q0 = (w.qgrp * a.rows_g + r) % N, i_q1 = (w.qgrp * a.rows_g + 128 + r) % N;   // pseudo-query indices
+    if (kFold) {
+      // The [256 x 16] operand: row i holds -r_i as an fp16 pair in channels 0 and 1 (zeros elsewhere, also
+      // for rows beyond the group); the operand of ones carries its two ones in BOTH 16-byte halves of every
+      // row, so whichever way the 32-byte swizzle orders the halves, the k-step adds exactly hi + lo.
+      const int te = (warp - kFirstEpiWarp) * 32 + lane;        // 0 .. 511
+      const float* ref = a.ref + w.qrow_base + w.qgrp * a.rows_g;
+      auto split = [&](int row, uint32_t& pair) -> float {      // the reference as the MMAs will see it
+        if (row >= w.rows) { pair = 0u; return 0.f; }
+        const float l = -ref[row];
+        const __half hi = __float2half_rn(l), lo = __float2half_rn(l - __half2float(hi));
+        pair = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+        return -(__half2float(hi) + __half2float(lo));
+      };
+      if (te < kGroupRows) {
+        uint32_t pair;
+        split(te, pair);
+        const uint32_t dst = sbase + kRefSlab + (te >> 3) * 256 + (te & 7) * 32;
+        sts128(dst, make_uint4(pair, 0u, 0u, 0u));
+        sts128(dst + 16, make_uint4(0u, 0u, 0u, 0u));
+      }
+      if (te < kOnes1SlabBytes / 16) sts128(sbase + Smem::exch + te * 16, make_uint4(0x3c003c00u, 0u, 0u, 0u));
+      fence_proxy_async();                                      // the MMAs read both operands through the async proxy
+      uint32_t unused;
+      rs0.init(split(r, unused));
+      rs1.init(split(128 + r, unused));
+      epilogue_sync();
+      if (warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());
+    }
     for (int ti = 0; ti < nt && ok; ++ti) {
       const int tile_base = (w.t0 + ti) * kTile1;
       const bool masked = tile_base + kTile1 > L;               // holds synthetic (or foreign) rows
@@ -170,7 +253,15 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.acc_empty(buf));
         // key column `col` of this tile is visible to pseudo query i iff its position <= L + i
-        if (m == 0) {
+        if (kFold) {
+          if (m == 0) {
+            if (masked) row_sum_cols<true>(v, col0, L + i_q0 - tile_base, rs0);
+            else row_sum_cols<false>(v, col0, 0, rs0);
+          } else {
+            if (masked) row_sum_cols<true>(v, col0, L + i_q1 - tile_base, rs1);
+            else row_sum_cols<false>(v, col0, 0, rs1);
+          }
+        } else if (m == 0) {
           if (masked) row_stats_cols<true>(v, col0, L + i_q0 - tile_base, c, m_raw0, z0);
           else row_stats_cols<false>(v, col0, 0, c, m_raw0, z0);
         } else {
@@ -182,7 +273,8 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // The four groups hold the statistics of the same rows over different key columns: group 3 puts its
     // pair into shared memory, groups 2 and 1 fold theirs in, group 0 folds last and stores the chunk's
     // partials (a fixed order, so the result does not depend on timing).
-    float2 s0 = make_float2(m_raw0 * c, z0), s1 = make_float2(m_raw1 * c, z1);
+    float2 s0 = kFold ? make_float2(rs0.m, rs0.z) : make_float2(m_raw0 * c, z0);
+    float2 s1 = kFold ? make_float2(rs1.m, rs1.z) : make_float2(m_raw1 * c, z1);
 #pragma unroll
     for (int g = kEpiGroups - 1; g >= 0; --g) {
       if (eg == g) {

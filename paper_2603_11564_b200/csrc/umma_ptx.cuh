@@ -183,9 +183,16 @@ __device__ __forceinline__ float ex2(float x) {
 #endif
 constexpr uint32_t kPolyPairMask = DAPQ_POLY_PAIR_MASK;   // bit p: pair p of a 32-column piece takes the polynomial
 __device__ __forceinline__ float2 ex2_pair_mufu(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+// kSat: inputs above 128 give 2^128-ish values (> 1.7e38) instead of wrapping the exponent field, for callers
+// that detect overflow by the size of the result.
+template <bool kSat = false>
 __device__ __forceinline__ float2 ex2_pair_poly(float2 x) {
   x.x = fmaxf(x.x, -125.f);
   x.y = fmaxf(x.y, -125.f);
+  if (kSat) {
+    x.x = fminf(x.x, 128.f);
+    x.y = fminf(x.y, 128.f);
+  }
   const float2 magic = make_float2(12582912.f, 12582912.f), neg_magic = make_float2(-12582912.f, -12582912.f);
   const float2 t = __fadd2_rn(x, magic);
   const float2 n = __fadd2_rn(t, neg_magic);

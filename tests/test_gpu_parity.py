@@ -757,3 +757,25 @@ def test_wait_limit_gives_up_reports_timeout_and_recovers(dq, flags):
     np.testing.assert_array_equal(again["idx"], good["idx"])
     _check_evict(w, data, again, ref)
     dq.dapq_destroy(ctx)
+
+
+# --------------------------------------------------- logits far from the row's reference (sweep 1)
+@pytest.mark.parametrize("where", [3, 700, 1290])
+def test_logits_far_above_and_below_the_first_key(dq, where):
+    """Sweep 1 measures every logit of a row against the row's logit for the first key of the sequence and sums
+    2^(difference) without tracking a maximum; a key whose logit lies more than the float range above that
+    reference has to take the careful per-job path.  One key aligned with a query (logit about +150 for that
+    row, tens above or below the bulk for the others), early, in the middle and among the last tiles."""
+    w = _small(lens=(1300,), keep=(40,), n_q_heads=8, n_kv_heads=2, n_pseudo=64, n_needles=0, outlier_channels=0)
+    data = gi.draw_layer(w, 0, "cpu")
+    q_rot = util.oracle_q_rot(w, data)[0]                               # [H_q, N, d] float64
+    for h in range(w.n_kv_heads):
+        u = q_rot[h * w.group + 1, 7]
+        data["k"][h, where] = (150.0 * np.sqrt(128.0) * u / (u.norm() ** 2)).to(torch.bfloat16)
+    ref = util.oracle_evict(w, data)
+    lg = (q_rot[1] @ data["k"][0].double().T) / np.sqrt(128.0)
+    assert float(lg[7, where] - lg[7, 0]) > 120.0                        # beyond 2^127 in base 2 for that row
+    for flags in (0, dq.DAPQ_FLAG_Q_LO_SWEEP1 | dq.DAPQ_FLAG_Q_LO_SWEEP2):
+        ctx = _ctx(dq, w, flags=flags)
+        _check_evict(w, data, _gpu_evict(dq, w, data, ctx), ref)
+        dq.dapq_destroy(ctx)
