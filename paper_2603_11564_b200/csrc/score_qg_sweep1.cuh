@@ -18,6 +18,11 @@ namespace dapq {
 namespace qg {
 
 constexpr int kCols1 = kTile1 / kEpiGroups;    // key columns of a job per epilogue group
+// Column pairs of a job that take the polynomial exp2 when the sums run without a maximum: none.  That
+// path has so few instructions per element left that its exponentials all fit the MUFU pipe beside the MMAs
+// (measured: 348 / 357 / 359 / 371 us per launch with 0 / 1/8 / 1/4 / 3/8 of the pairs on the polynomial,
+// Llama-3-70B shape).
+constexpr uint32_t kPolyPairMaskSum = 0x0000u;
 
 // Running max / sum of exp over this thread's 48 columns of an accumulator row.
 // lim: last visible column of the tile for this thread's pseudo query (masked tiles only).
@@ -98,8 +103,8 @@ __device__ __forceinline__ void row_sum_cols(uint32_t* v, int col0, int lim, Row
 #pragma unroll
     for (int e = 0; e < kCols1; e += 4) {
       const float2 x0 = make_float2(x[e], x[e + 1]), x1 = make_float2(x[e + 2], x[e + 3]);
-      acc0 = __fadd2_rn(acc0, ((kPolyPairMask >> ((e / 2) & 15)) & 1u) ? ex2_pair_poly<true>(x0) : ex2_pair_mufu(x0));
-      acc1 = __fadd2_rn(acc1, ((kPolyPairMask >> ((e / 2 + 1) & 15)) & 1u) ? ex2_pair_poly<true>(x1) : ex2_pair_mufu(x1));
+      acc0 = __fadd2_rn(acc0, ((kPolyPairMaskSum >> ((e / 2) & 15)) & 1u) ? ex2_pair_poly<true>(x0) : ex2_pair_mufu(x0));
+      acc1 = __fadd2_rn(acc1, ((kPolyPairMaskSum >> ((e / 2 + 1) & 15)) & 1u) ? ex2_pair_poly<true>(x1) : ex2_pair_mufu(x1));
     }
     const float zj = (acc0.x + acc0.y) + (acc1.x + acc1.y);
     if (zj < 1e37f) {                                           // (false for inf and NaN too)
