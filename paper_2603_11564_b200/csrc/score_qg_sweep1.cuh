@@ -18,11 +18,14 @@ namespace dapq {
 namespace qg {
 
 constexpr int kCols1 = kTile1 / kEpiGroups;    // key columns of a job per epilogue group
-// Column pairs of a job that take the polynomial exp2 when the sums run without a maximum: none.  That
-// path has so few instructions per element left that its exponentials all fit the MUFU pipe beside the MMAs
-// (measured: 348 / 357 / 359 / 371 us per launch with 0 / 1/8 / 1/4 / 3/8 of the pairs on the polynomial,
-// Llama-3-70B shape).
-constexpr uint32_t kPolyPairMaskSum = 0x0000u;
+// Column pairs of a job that take the polynomial exp2 when the sums run without a maximum: none.  That path
+// has so few instructions per element left that it runs at the pace of the MUFU pipe either way (measured on
+// the Llama-3-70B shape: 0, 1/8 and 1/4 of the pairs on the polynomial are within 2 % of one another, in
+// both directions from one GPU to the next), so it keeps the simplest form.
+#ifndef DAPQ_POLY_PAIR_MASK_SUM
+#define DAPQ_POLY_PAIR_MASK_SUM 0x0000u
+#endif
+constexpr uint32_t kPolyPairMaskSum = DAPQ_POLY_PAIR_MASK_SUM;
 
 // Running max / sum of exp over this thread's 48 columns of an accumulator row.
 // lim: last visible column of the tile for this thread's pseudo query (masked tiles only).
