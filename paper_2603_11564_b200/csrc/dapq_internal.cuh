@@ -170,7 +170,8 @@ cudaError_t launch_score_umma(const UmmaPlan& plan, const SeqTable& t, const Dim
 // the sequences' keys into chunks of whole tiles with ctas_per_chunk CTAs working on every chunk.
 bool encode_tile_map(CUtensorMap* map, const void* base, bool f16, int rank, const uint64_t* dims,
                      const uint64_t* strides_bytes, int box_rows);
-bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_chunk, int n_sm, ChunkTable* ct);
+bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_chunk, int n_sm, ChunkTable* ct,
+                 double cta_cost = 3.0);
 
 // Tensor-core scorer with one query group per CTA (score_qg.cu).  q: [B*H_q*N, d], fp16 (the K tiles
 // are then converted to fp16 in shared memory) or bf16.  qg_plan returns false when the view cannot be

@@ -100,8 +100,10 @@ bool encode_tile_map(CUtensorMap* map, const void* base, bool f16, int rank, con
 }
 
 // Cut every sequence's keys (prompt, plus the synthetic rows if asked) into chunks of whole tiles;
-// ctas_per_chunk CTAs work on every chunk (KV heads x query groups).
-bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_chunk, int n_sm, ChunkTable* ct) {
+// ctas_per_chunk CTAs work on every chunk (KV heads x query groups).  cta_cost: what a CTA spends besides
+// its tiles (set-up, first loads, drain), in units of one tile's work.
+bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_chunk, int n_sm, ChunkTable* ct,
+                 double cta_cost) {
   int max_tiles = 0;
   for (int b = 0; b < t.batch; ++b) {
     const int tiles = (t.prompt_len[b] + extra_keys + tile_keys - 1) / tile_keys;
@@ -118,7 +120,7 @@ bool plan_chunks(const SeqTable& t, int extra_keys, int tile_keys, int ctas_per_
     }
     if (n > t.batch + kUmmaMaxChunks) continue;
     const int64_t waves = (n * ctas_per_chunk + n_sm - 1) / n_sm;
-    const double cost = (double)waves * (c + 3.0);
+    const double cost = (double)waves * (c + cta_cost);
     if (best_c == 0 || cost < best_cost) { best_c = c; best_cost = cost; }
   }
   if (best_c == 0) return false;
@@ -147,8 +149,10 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
   plan->n_stages1 = s1 < kMaxStages ? s1 : kMaxStages;
   plan->n_stages2 = s2 < kMaxStages ? s2 : kMaxStages;
   const int ctas = dm.n_kv_heads * plan->n_qgroups;
-  if (!plan_chunks(t, dm.n_pseudo, kTile1, ctas, n_sm, &plan->ct1)) return false;
-  if (!plan_chunks(t, 0, kTile2, ctas, n_sm, &plan->ct2)) return false;
+  // (a sweep-2 tile is one job of about a microsecond, a sweep-1 tile two: a CTA's set-up of several
+  // microseconds weighs more tiles in sweep 2, where ragged batches would otherwise be cut into waves of short CTAs)
+  if (!plan_chunks(t, dm.n_pseudo, kTile1, ctas, n_sm, &plan->ct1, 3.0)) return false;
+  if (!plan_chunks(t, 0, kTile2, ctas, n_sm, &plan->ct2, 6.0)) return false;
   // ---- tensor maps: K as [d, rows, H_kv] (one map per sweep: the boxes differ), the query operand as [d, rows]
   const uint64_t rows_k = (uint64_t)t.cu_rows[t.batch];
   const uint64_t kd[3] = {(uint64_t)kHeadDim, rows_k, (uint64_t)dm.n_kv_heads};
