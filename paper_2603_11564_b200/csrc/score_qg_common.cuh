@@ -184,7 +184,12 @@ __device__ __forceinline__ void cta_epilogue(uint32_t tmem_base) {
 // ---- TMA producer (one thread): the first K tile, the CTA's query group, then the rest of the ring.
 // Returns only when every copy it issued has landed (also when the CTA is aborting), so that the CTA
 // never exits with a copy into its shared memory in flight.
-template <int kTile>
+// kGate (sweep 2): the tiles after the first wait until the epilogue warps have read sweep 1's partials.  At
+// the start of a launch every SM asks for its whole ring at once; whatever is queued behind those copies,
+// the small loads of the partials among it, then takes microseconds to arrive, and the first job cannot
+// start without them (measured on the 32k shape: first MMA 8400 cycles after CTA entry, partials 5000 cycles
+// in flight).
+template <int kTile, bool kGate = false>
 __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w, const Args& a,
                                              uint32_t sbase, const Bars& bars, int kvh, const Waiter& wt) {
   using T = TileGeo<kTile>;
@@ -207,6 +212,7 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     for (int m = 0; m < w.mb; ++m)
       tma_load_2d(sbase + half * (q_bytes / 2) + m * 128 * 128, tm_q, bars.q_full(), half * 64,
                   w.qrow_base + w.qgrp * a.rows_g + m * 128);
+  if (kGate) ok = wt.wait(bars.lse_ready(), 0);
   Ring rs(S);
   for (int ti = 1; ti < w.nt && ok; ++ti) {
     rs.next();

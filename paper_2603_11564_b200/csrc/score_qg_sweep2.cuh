@@ -108,7 +108,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
   const int S = a.n_stages;
 
   if (warp == 0) {
-    if (lane == 0) tma_producer<kTile2>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+    if (lane == 0) tma_producer<kTile2, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
@@ -212,7 +212,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         fence_proxy_async();                                    // the MMAs read both operands through the async proxy
       }
       epilogue_sync();
-      if (kFold && warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());
+      if (warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());    // (the MMA issuer and the TMA producer wait for it)
     }
     // Pieces of a job (16 query columns): group g takes pieces [g nch / 4, (g + 1) nch / 4), at most four
     const int nch = ncols >> 4;
