@@ -218,9 +218,9 @@ dapq_status run_score_umma(dapq_ctx* ctx, const UmmaPlan& plan, const SeqTable& 
 }
 
 dapq_status run_score_qg(dapq_ctx* ctx, const QgPlan& plan, const SeqTable& t, const float* lse_in,
-                         float* scores, int64_t score_stride, float* lse_out, cudaStream_t s) {
+                         float* scores, int64_t score_stride, float* lse_out, bool after_rope, cudaStream_t s) {
   cudaError_t e = launch_score_qg(plan, t, ctx->dims, lse_in, ctx->part, ctx->slots, scores, score_stride, lse_out,
-                                  ctx->lse2, ctx->status, ctx->wait_limit, s, &ctx->log);
+                                  ctx->lse2, ctx->status, ctx->wait_limit, after_rope, s, &ctx->log);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tensor-core score kernels");
   return DAPQ_OK;
 }
@@ -470,7 +470,7 @@ dapq_status dapq_score(dapq_ctx* ctx, const void* q_rot, const dapq_cache_view* 
     } else {
       QgPlan plan;
       if (qg_plan(q_rot, 0, cd, t, ctx->dims, ctx->n_sm, &plan))
-        return run_score_qg(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, (cudaStream_t)stream);
+        return run_score_qg(ctx, plan, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, false, (cudaStream_t)stream);
     }
   }
   return run_score(ctx, ctx->shape.dtype, q_rot, cd, t, lse_in, scores, t.cu_prompt[t.batch], lse_out, syn_mass, (cudaStream_t)stream);
@@ -558,7 +558,7 @@ dapq_status evict_impl(dapq_ctx* ctx, const void* q_pre, const dapq_cache_view* 
     e = launch_rope(ctx->shape.dtype, qplan.q_is_f16 ? kRopeOutF16 : kRopeOutBf16, 0, q_pre, ctx->q_rot, ctx->inv_freq, t,
                     ctx->dims, after_own_compaction, s, &ctx->log, &ref);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rope kernel");
-    st = run_score_qg(ctx, qplan, t, nullptr, scores, score_stride, nullptr, s);
+    st = run_score_qg(ctx, qplan, t, nullptr, scores, score_stride, nullptr, true, s);
   } else if (wants_umma(ctx) && wants_lo(ctx) && umma_plan(ctx->q_rot, 1, lo_rows, cd, t, ctx->dims, ctx->n_sm, &plan)) {
     // older tensor-core scorer: rotated queries as a bf16 pair hi + lo, the lo part added by a second MMA
     // pass in the sweeps that the flags name

@@ -185,9 +185,11 @@ struct QgPlan {
 int qg_groups(const Dims& dm);
 bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t, const Dims& dm, int n_sm, QgPlan* plan);
 // ref: with fp16 queries, the [B, H_q, N] reference logits that the rotation kernel wrote beside them.
+// after_own_kernel: the kernel before these in the stream is this library's rotation kernel (which waits for
+// whatever precedes it), so the sweeps may copy the keys before their own wait for it.
 cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in, float2* part,
                             float* slots, float* scores, int64_t score_stride, float* lse_out, const float* ref, int* status,
-                            long long wait_limit, cudaStream_t s, LaunchLog* log);
+                            long long wait_limit, bool after_own_kernel, cudaStream_t s, LaunchLog* log);
 
 cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx, int64_t idx_stride,
                         const SeqTable& t, int n_kv_heads, cudaStream_t s, LaunchLog* log);

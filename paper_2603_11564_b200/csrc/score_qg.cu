@@ -168,7 +168,7 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
 
 cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& dm, const float* lse_in, float2* part,
                             float* slots, float* scores, int64_t score_stride, float* lse_out, const float* ref, int* status,
-                            long long wait_limit, cudaStream_t s, LaunchLog* log) {
+                            long long wait_limit, bool after_own_kernel, cudaStream_t s, LaunchLog* log) {
   Args a;
   a.n_pseudo = dm.n_pseudo;
   a.group = dm.group;
@@ -195,6 +195,7 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
     if ((e = cudaFuncSetAttribute(sweep2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
     if (lse_in == nullptr) {
       a.n_stages = plan.n_stages1;
+      a.early_loads = after_own_kernel ? 1 : 0;
       log->begin(kKindSweep1, s);
       e = launch_pdl(sweep1, dim3(plan.ct1.n_chunks * plan.n_qgroups, dm.n_kv_heads), dim3(kThreads1), kSmemBytes, s, 1,
                      plan.tm_k1, plan.tm_q, t, plan.ct1, a);
@@ -202,6 +203,7 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
       if (e != cudaSuccess) return e;
     }
     a.n_stages = plan.n_stages2;
+    a.early_loads = (after_own_kernel || lse_in == nullptr) ? 1 : 0;     // (sweep 1, if it ran, waited for what came before)
     log->begin(kKindSweep2, s);
     e = launch_pdl(sweep2, dim3(plan.ct2.n_chunks * plan.n_qgroups, dm.n_kv_heads), dim3(kThreads2), kSmemBytes, s, 1,
                    plan.tm_k2, plan.tm_q, t, plan.ct2, plan.ct1, a);

@@ -63,6 +63,8 @@ struct Args {
   int32_t rows_g;            // rows per group (a multiple of 16; the last group may hold fewer)
   int32_t rows_pad;          // row pitch of `part`
   int32_t n_stages;          // K stages that fit beside the group's queries
+  int32_t early_loads;       // the kernel before this one in the stream is one of this library's that waited for ITS
+                             // predecessor: inputs it does not write may be copied before this kernel's own wait
   float scale_log2e;
   long long wait_limit;      // cycles a wait may take before the CTA gives up
   float2* part;              // [n_chunks1, H_kv, rows_pad] (running max, sum) of every query row over a chunk's keys, base 2
@@ -135,30 +137,29 @@ struct Waiter {
   __device__ __forceinline__ bool aborting() const { return *abort_flag != 0; }
 };
 
-// Common CTA prologue: barrier init, tensor-memory allocation (warp 1), one CTA-wide sync, then
-// the wait for the kernel before this one (its set-up overlaps that kernel's tail).
-// Returns the tensor-memory base address.
-__device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars) {
-  const int warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(bars.k_full(s), 1);
-      mbar_init(bars.k_conv(s), kConvWarps);
-      mbar_init(bars.k_empty(s), 1);
-    }
-    for (int i = 0; i < kMaxAcc; ++i) {
-      mbar_init(bars.acc_full(i), 1);
-      mbar_init(bars.acc_empty(i), 4 * kEpiGroups);        // every epilogue warp reads every accumulator
-    }
-    for (int i = 0; i < kExchDepth; ++i) {
-      mbar_init(bars.part_full(i), 4 * kEpiGroups);        // every epilogue warp posts its partial sums
-      mbar_init(bars.part_empty(i), 1);                    // the summing warp has read them
-    }
-    mbar_init(bars.q_full(), 1);
-    mbar_init(bars.drain(), 1);
-    mbar_init(bars.lse_ready(), 1);
-    *reinterpret_cast<volatile int*>(smem + Smem::abort_flag) = 0;
+// Arrivals that complete a phase of barrier `idx` (in the order of Bars).
+__device__ __forceinline__ uint32_t bar_count(int idx) {
+  if (idx < kMaxStages) return 1u;                                        // k_full: the producer (+ the copies' bytes)
+  if (idx < 2 * kMaxStages) return kConvWarps;                            // k_conv
+  if (idx < 3 * kMaxStages + kMaxAcc) return 1u;                          // k_empty, acc_full: one tcgen05.commit
+  if (idx < 3 * kMaxStages + 2 * kMaxAcc + kExchDepth) return 4u * kEpiGroups;   // acc_empty, part_full: every epilogue warp
+  return 1u;                                                              // part_empty, q_full, drain, lse_ready
+}
+
+// Common CTA prologue: barrier init (warp 0, one barrier per lane), the first TMA copies (`first`, run by
+// thread 0 as soon as the barriers exist: only copies of data that the kernel before this one does not
+// write), tensor-memory allocation (warp 1), one CTA-wide sync, then the wait for the kernel before this one
+// (all of this overlaps that kernel's tail).  Returns the tensor-memory base address.
+template <class First>
+__device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, First first) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  static_assert(Smem::n_bars <= 32, "one barrier per lane of warp 0");
+  if (warp == 0) {
+    if (lane < Smem::n_bars) mbar_init(bars.base + 8u * lane, bar_count(lane));
+    if (lane == 0) *reinterpret_cast<volatile int*>(smem + Smem::abort_flag) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) first();
   }
   if (warp == 1) {                                              // tensor memory: all 512 columns
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -168,7 +169,7 @@ __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  pdl_wait();                                                   // global memory is touched only from here on
+  pdl_wait();                                                   // what the previous kernel wrote is read only from here on
   return *reinterpret_cast<volatile uint32_t*>(smem + Smem::tmem_ptr);
 }
 
@@ -181,22 +182,41 @@ __device__ __forceinline__ void cta_epilogue(uint32_t tmem_base) {
   }
 }
 
-// ---- TMA producer (one thread): the first K tile, the CTA's query group, then the rest of the ring.
-// Returns only when every copy it issued has landed (also when the CTA is aborting), so that the CTA
-// never exits with a copy into its shared memory in flight.
-// kGate (sweep 2): the tiles after the first wait until the epilogue warps have read sweep 1's partials.  At
-// the start of a launch every SM asks for its whole ring at once; whatever is queued behind those copies,
-// the small loads of the partials among it, then takes microseconds to arrive, and the first job cannot
-// start without them (measured on the 32k shape: first MMA 8400 cycles after CTA entry, partials 5000 cycles
-// in flight).
-template <int kTile, bool kGate = false>
+// ---- TMA producer (one thread).  tma_first issues the first K tile and, if the queries are not written by
+// the kernel before this one (kWithQ), the CTA's query group; it runs inside the prologue.  tma_producer
+// then issues the queries if they are still owed and the rest of the ring.  It returns only when every copy
+// has landed (also when the CTA is aborting), so that the CTA never exits with a copy into its shared
+// memory in flight.
+__device__ __forceinline__ void tma_queries(const CUtensorMap* tm_q, const Work& w, const Args& a, uint32_t sbase, const Bars& bars) {
+  const uint32_t q_bytes = (uint32_t)w.mb * 2u * 128u * 128u;
+  mbar_expect_tx(bars.q_full(), q_bytes);
+  for (int half = 0; half < 2; ++half)
+    for (int m = 0; m < w.mb; ++m)
+      tma_load_2d(sbase + half * (q_bytes / 2) + m * 128 * 128, tm_q, bars.q_full(), half * 64,
+                  w.qrow_base + w.qgrp * a.rows_g + m * 128);
+}
+template <int kTile, bool kWithQ>
+__device__ __forceinline__ void tma_first(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w, const Args& a,
+                                          uint32_t sbase, const Bars& bars, int kvh) {
+  using T = TileGeo<kTile>;
+  const uint32_t ring = sbase + (uint32_t)w.mb * 2u * 128u * 128u;
+  mbar_expect_tx(bars.k_full(0), T::kStage);                // (w.nt >= 1: checked by the caller)
+  const int row = w.row_base + w.t0 * kTile;
+  tma_load_3d(ring, tm_k, bars.k_full(0), 0, row, kvh);
+  tma_load_3d(ring + T::kHalf, tm_k, bars.k_full(0), 64, row, kvh);
+  if (kWithQ) tma_queries(tm_q, w, a, sbase, bars);
+}
+// kQOwed: the queries were not part of tma_first.  kGate (sweep 2): the tiles after the first wait until the
+// epilogue warps have merged sweep 1's partials: at the start of a launch every SM asks for its whole ring at
+// once, and whatever is queued behind those copies takes microseconds to arrive.
+template <int kTile, bool kQOwed, bool kGate>
 __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUtensorMap* tm_q, const Work& w, const Args& a,
                                              uint32_t sbase, const Bars& bars, int kvh, const Waiter& wt) {
   using T = TileGeo<kTile>;
   const int S = a.n_stages;
   const uint32_t q_bytes = (uint32_t)w.mb * 2u * 128u * 128u;
   const uint32_t ring = sbase + q_bytes;
-  int li = 0;                                               // K tiles issued so far
+  int li = 1;                                               // K tiles issued so far (the first by tma_first)
   bool ok = true;
   auto load_tile = [&](int ti) {
     const int s = li % S;                                   // (li == ti; one division per tile in this single thread)
@@ -206,12 +226,7 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     tma_load_3d(ring + s * T::kStage + T::kHalf, tm_k, bars.k_full(s), 64, row, kvh);
     ++li;
   };
-  load_tile(0);                                             // (w.nt >= 1: checked by the caller)
-  mbar_expect_tx(bars.q_full(), q_bytes);
-  for (int half = 0; half < 2; ++half)
-    for (int m = 0; m < w.mb; ++m)
-      tma_load_2d(sbase + half * (q_bytes / 2) + m * 128 * 128, tm_q, bars.q_full(), half * 64,
-                  w.qrow_base + w.qgrp * a.rows_g + m * 128);
+  if (kQOwed) tma_queries(tm_q, w, a, sbase, bars);
   if (kGate) ok = wt.wait(bars.lse_ready(), 0);
   Ring rs(S);
   for (int ti = 1; ti < w.nt && ok; ++ti) {

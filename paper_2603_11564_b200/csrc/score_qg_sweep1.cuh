@@ -150,12 +150,18 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   if (nt <= 0) return;
   const Bars bars{sbase + Smem::bars};
   const Waiter wt{reinterpret_cast<volatile int*>(smem + Smem::abort_flag), a.status, a.wait_limit};
-  const uint32_t tmem_base = cta_prologue(smem, sbase, bars);
+  // (the keys are nobody's output in this stream; the queries are the rotation kernel's, the kernel before)
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, [&] {
+    if (a.early_loads) tma_first<kTile1, false>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
+  });
   const uint32_t q_half = (uint32_t)mb * 128u * 128u;           // bytes of one 64-channel half of the query group
   const int S = a.n_stages;
 
   if (warp == 0) {
-    if (lane == 0) tma_producer<kTile1>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+    if (lane == 0) {
+      if (!a.early_loads) tma_first<kTile1, false>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
+      tma_producer<kTile1, true, false>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+    }
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {

@@ -101,14 +101,37 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
   float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
   float* aux = reinterpret_cast<float*>(smem + Smem::aux);      // [256] scratch of the lse merge
   float* exch = reinterpret_cast<float*>(smem + Smem::exch);    // [kExchDepth][4][128] partial sums on their way to the summing warp
-  const uint32_t tmem_base = cta_prologue(smem, sbase, bars);
+  // The epilogue threads ask for sweep 1's partials of their query row first of all, before the CTA's copies of
+  // queries and keys crowd the memory system (two threads per row: thread (eg, r) takes row (eg & 1) * 128 + r and
+  // the chunks of parity eg >> 1; up to 16 partials per thread at once).
+  const bool is_epi = warp >= kFirstEpiWarp && warp < kFirstEpiWarp + 4 * kEpiGroups;
+  const int m_eg = (warp - kFirstEpiWarp) >> 2, m_row = (m_eg & 1) * 128 + (warp & 3) * 32 + lane;
+  const bool m_live = is_epi && m_row < w.rows && !a.lse_in;
+  const int m_nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
+  const int64_t m_step = (int64_t)a.n_kv_heads * a.rows_pad;
+  const float2* m_p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * a.rows_pad + w.qgrp * a.rows_g + m_row;
+  float2 m_q[16];
+  if (m_live) {
+    pdl_wait();                                                 // (sweep 1 wrote them)
+#pragma unroll
+    for (int u = 0; u < 16; ++u)
+      m_q[u] = (m_eg >> 1) + 2 * u < m_nc ? __ldg(m_p + ((m_eg >> 1) + 2 * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
+  }
+  // (behind this library's own sweep 1 or rotation kernel, keys and queries were complete before that kernel
+  // got past its wait: both go out at once)
+  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, [&] {
+    if (a.early_loads) tma_first<kTile2, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
+  });
   const int ncols = (w.rows + 15) & ~15;                        // UMMA N: only the query columns that exist
   const int acc_cols = ncols > 128 ? 256 : 128, n_acc = kTmemCols / acc_cols;
   const uint32_t q_half = (uint32_t)w.mb * 128u * 128u;         // bytes of one 64-channel half of the query group
   const int S = a.n_stages;
 
   if (warp == 0) {
-    if (lane == 0) tma_producer<kTile2, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+    if (lane == 0) {
+      if (!a.early_loads) tma_first<kTile2, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
+      tma_producer<kTile2, false, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh, wt);
+    }
   } else if (warp == 1) {
     // ============================================================================= MMA issuer
     if (lane == 0) {
@@ -154,25 +177,23 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
       const int row = (eg & 1) * 128 + r, grow = w.qgrp * a.rows_g + row;
       const bool live = row < w.rows;
       float mx = -CUDART_INF_F, z = 0.f;
-      if (live && !a.lse_in) {
-        const float2* p = a.part + ((int64_t)ct1.cu_chunk[b] * a.n_kv_heads + kvh) * a.rows_pad + grow;
-        const int64_t step = (int64_t)a.n_kv_heads * a.rows_pad;
-        const int nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
-        for (int c0 = eg >> 1; c0 < nc; c0 += 32) {
-          float2 q[16];
+      if (m_live) {
+        for (int c0 = eg >> 1; c0 < m_nc; c0 += 32) {
+          if (c0 > (eg >> 1)) {                                 // (more than 32 chunks: the next batch)
 #pragma unroll
-          for (int u = 0; u < 16; ++u)
-            q[u] = c0 + 2 * u < nc ? __ldg(p + (c0 + 2 * u) * step) : make_float2(-CUDART_INF_F, 0.f);
-          float m16 = q[0].x;
+            for (int u = 0; u < 16; ++u)
+              m_q[u] = c0 + 2 * u < m_nc ? __ldg(m_p + (c0 + 2 * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
+          }
+          float m16 = m_q[0].x;
 #pragma unroll
-          for (int u = 1; u < 16; ++u) m16 = fmaxf(m16, q[u].x);
+          for (int u = 1; u < 16; ++u) m16 = fmaxf(m16, m_q[u].x);
           if (m16 > mx) {
             z *= exp2f(mx - m16);                               // exp2f(-inf) = 0 on the first round
             mx = m16;
           }
           if (mx > -CUDART_INF_F) {
 #pragma unroll
-            for (int u = 0; u < 16; ++u) z += q[u].y * exp2f(q[u].x - mx);
+            for (int u = 0; u < 16; ++u) z += m_q[u].y * exp2f(m_q[u].x - mx);
           }
         }
       }
