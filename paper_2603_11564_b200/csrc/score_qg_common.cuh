@@ -226,7 +226,11 @@ __device__ __forceinline__ void tma_producer(const CUtensorMap* tm_k, const CUte
     tma_load_3d(ring + s * T::kStage + T::kHalf, tm_k, bars.k_full(s), 64, row, kvh);
     ++li;
   };
-  if (kQOwed) tma_queries(tm_q, w, a, sbase, bars);
+  if (kQOwed) {
+    // (the first job needs the queries, not the tiles after the first: those go out once the queries are in)
+    tma_queries(tm_q, w, a, sbase, bars);
+    ok = wt.wait(bars.q_full(), 0);
+  }
   if (kGate) ok = wt.wait(bars.lse_ready(), 0);
   Ring rs(S);
   for (int ti = 1; ti < w.nt && ok; ++ti) {

@@ -150,6 +150,18 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   if (nt <= 0) return;
   const Bars bars{sbase + Smem::bars};
   const Waiter wt{reinterpret_cast<volatile int*>(smem + Smem::abort_flag), a.status, a.wait_limit};
+  // With reference logits: the epilogue threads ask for theirs first of all (the rotation kernel, the kernel before
+  // this one, wrote them), before the CTA's copies of keys and queries crowd the memory system: row te of the
+  // [256 x 16] operand, and the thread's own two accumulator rows.
+  float ref_slab = 0.f, ref_r0 = 0.f, ref_r1 = 0.f;
+  if (kFold && warp >= kFirstEpiWarp) {
+    pdl_wait();
+    const float* ref = a.ref + w.qrow_base + w.qgrp * a.rows_g;
+    const int te = (warp - kFirstEpiWarp) * 32 + lane, r_ = (warp & 3) * 32 + lane;
+    if (te < w.rows) ref_slab = __ldg(ref + te);
+    if (r_ < w.rows) ref_r0 = __ldg(ref + r_);
+    if (128 + r_ < w.rows) ref_r1 = __ldg(ref + 128 + r_);
+  }
   // (the keys are nobody's output in this stream; the queries are the rotation kernel's, the kernel before)
   const uint32_t tmem_base = cta_prologue(smem, sbase, bars, [&] {
     if (a.early_loads) tma_first<kTile1, false>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
@@ -222,17 +234,16 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // for rows beyond the group); the operand of ones carries its two ones in BOTH 16-byte halves of every
       // row, so whichever way the 32-byte swizzle orders the halves, the k-step adds exactly hi + lo.
       const int te = (warp - kFirstEpiWarp) * 32 + lane;        // 0 .. 511
-      const float* ref = a.ref + w.qrow_base + w.qgrp * a.rows_g;
-      auto split = [&](int row, uint32_t& pair) -> float {      // the reference as the MMAs will see it
+      auto split = [&](int row, float ref_val, uint32_t& pair) -> float {   // the reference as the MMAs will see it
         if (row >= w.rows) { pair = 0u; return 0.f; }
-        const float l = -ref[row];
+        const float l = -ref_val;
         const __half hi = __float2half_rn(l), lo = __float2half_rn(l - __half2float(hi));
         pair = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
         return -(__half2float(hi) + __half2float(lo));
       };
       if (te < kGroupRows) {
         uint32_t pair;
-        split(te, pair);
+        split(te, ref_slab, pair);
         const uint32_t dst = sbase + kRefSlab + (te >> 3) * 256 + (te & 7) * 32;
         sts128(dst, make_uint4(pair, 0u, 0u, 0u));
         sts128(dst + 16, make_uint4(0u, 0u, 0u, 0u));
@@ -240,8 +251,8 @@ rowstat_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (te < kOnes1SlabBytes / 16) sts128(sbase + Smem::exch + te * 16, make_uint4(0x3c003c00u, 0u, 0u, 0u));
       fence_proxy_async();                                      // the MMAs read both operands through the async proxy
       uint32_t unused;
-      rs0.init(split(r, unused));
-      rs1.init(split(128 + r, unused));
+      rs0.init(split(r, ref_r0, unused));
+      rs1.init(split(128 + r, ref_r1, unused));
       epilogue_sync();
       if (warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());
     }
