@@ -30,7 +30,8 @@ constexpr int kKeysPerCta = 4096;             // a CTA owns about this many keys
 constexpr int kWaveCtas = 296;                // when the grid would otherwise exceed one wave (2 CTAs per SM)
 constexpr int kBins = 2048;                   // 11-bit digits (the last pass uses 1024 of them)
 constexpr int kMaxSliceSmem = 36864;          // keys a CTA can cache (144 KB); longer slices re-read global
-constexpr int kMaxCand = 4096;                // candidate keys a CTA lists after the first pass
+constexpr int kMaxCand = 4096;                // candidate keys a CTA lists after the first pass (general kernel)
+constexpr int kRegion = 2048;                 // candidate keys per CTA that the keys-in-registers kernel exchanges
 
 // Monotone map float -> uint32 (larger float <=> larger key), valid for all finite values.
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -38,40 +39,59 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-struct TopkSmem {
+struct TopkTables {
   uint32_t merged[3][kBins];   // cluster-wide histogram of each pass (every CTA holds a copy)
   uint32_t hist[kBins];        // this CTA's histogram (all zero between passes)
-  uint32_t cand[kMaxCand];     // this CTA's keys that share the first pass's digit
   uint32_t warp_sum[kWarps];
   uint32_t cnt_gt[kWarps], cnt_eq[kWarps];
   uint32_t peer_gt[kCluster], peer_eq[kCluster];   // totals of every CTA of the cluster, pushed by their owners
-  uint32_t prefix, remaining, n_cand, list_ok;
+  uint32_t prefix, remaining, n_cand, own_count;
 };
 
-// Adds this CTA's non-empty bins into the merged table of every CTA of the cluster and leaves the local table
-// clear; local_bins keeps the thread's own two counts (the first pass's decide whether the candidates fit the list).
-__device__ __forceinline__ void push_bins(TopkSmem& sm, uint32_t* const (&peer_merged)[kCluster], int n_cta, int pass,
-                                          int tid, uint32_t (&local_bins)[kBins / kTopkThreads]) {
+struct TopkSmem {              // general kernel; the cached keys follow
+  TopkTables tb;
+  uint32_t cand[kMaxCand];     // this CTA's keys that share the first pass's digit
+};
+
+struct TopkRegSmem {           // keys-in-registers kernel
+  TopkTables tb;
+  uint32_t cand[kCluster][kRegion];   // the candidates of EVERY CTA of the cluster (each pushes its own to all)
+  uint32_t peer_cnt[kCluster];        // how many candidates CTA r has (more than kRegion: it pushed none)
+  uint32_t peer_hi[kCluster];         // how many keys of CTA r lie above the first pass's digit
+  uint32_t reg_gt[kCluster], reg_eq[kCluster];
+  uint32_t hi_own;
+};
+
+// Thread t owns digits 2047-2t and 2046-2t of every table.  Adds this CTA's non-empty bins into the merged
+// table of every CTA of the cluster and leaves the local table clear; local keeps the thread's own two counts.
+__device__ __forceinline__ void push_bins(TopkTables& tb, uint32_t* const (&peer_merged)[kCluster], int n_cta, int pass,
+                                          int tid, uint32_t (&local)[2]) {
+  const int d_hi = kBins - 1 - 2 * tid;
+  const uint2 c2 = *reinterpret_cast<const uint2*>(&tb.hist[d_hi - 1]);
+  local[0] = c2.y;
+  local[1] = c2.x;
+  if (c2.x | c2.y) {
+    *reinterpret_cast<uint2*>(&tb.hist[d_hi - 1]) = make_uint2(0u, 0u);
 #pragma unroll
-  for (int e = 0; e < kBins / kTopkThreads; ++e) {
-    const int d = tid + e * kTopkThreads;
-    const uint32_t c = sm.hist[d];
-    local_bins[e] = c;
-    if (c) {
-      sm.hist[d] = 0u;
+    for (int e = 0; e < 2; ++e) {
+      if (local[e]) {
 #pragma unroll
-      for (int p = 0; p < kCluster; ++p)
-        if (p < n_cta) atomicAdd(peer_merged[p] + pass * kBins + d, c);
+        for (int p = 0; p < kCluster; ++p)
+          if (p < n_cta) atomicAdd(peer_merged[p] + pass * kBins + d_hi - e, local[e]);
+      }
     }
   }
 }
 
-// Scans the merged table of `pass` from the top digit down for the digit that holds the K-th entry (thread t owns
-// digits 2047-2t and 2046-2t); extends sm.prefix by it and reduces sm.remaining to the rank within that digit.
-__device__ __forceinline__ void select_digit(TopkSmem& sm, int pass, int shift, uint32_t prefix, int tid, int lane, int warp) {
-  const uint32_t remaining = sm.remaining;
+// Scans `table` from the top digit down for the digit that holds the entry of rank tb.remaining; extends
+// tb.prefix by it, reduces tb.remaining to the rank within that digit and leaves this CTA's own count of the
+// digit in tb.own_count.  Every warp sums the totals of the warps before it by itself: two block barriers.
+__device__ __forceinline__ void select_digit(TopkTables& tb, const uint32_t* table, int shift, uint32_t prefix,
+                                             const uint32_t (&local)[2], int tid, int lane, int warp) {
+  const uint32_t remaining = tb.remaining;
   const int d_hi = kBins - 1 - 2 * tid;
-  const uint32_t v0 = sm.merged[pass][d_hi], v1 = sm.merged[pass][d_hi - 1];
+  const uint2 v = *reinterpret_cast<const uint2*>(&table[d_hi - 1]);
+  const uint32_t v0 = v.y, v1 = v.x;
   const uint32_t mine = v0 + v1;
   uint32_t incl = mine;
 #pragma unroll
@@ -79,34 +99,53 @@ __device__ __forceinline__ void select_digit(TopkSmem& sm, int pass, int shift, 
     const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += y;
   }
-  if (lane == 31) sm.warp_sum[warp] = incl;
+  if (lane == 31) tb.warp_sum[warp] = incl;
   __syncthreads();
-  if (warp == 0) {
-    const uint32_t ws = sm.warp_sum[lane];
-    uint32_t wi = ws;
+  uint32_t before = lane < warp ? tb.warp_sum[lane] : 0u;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    sm.warp_sum[lane] = wi - ws;                         // exclusive prefix of the warp sums
-  }
-  __syncthreads();
-  incl += sm.warp_sum[warp];
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+  incl += before;
   const uint32_t excl = incl - mine;
   if (excl < remaining && incl >= remaining) {           // exactly one thread
     const bool first = excl + v0 >= remaining;
-    sm.prefix = prefix | ((uint32_t)(first ? d_hi : d_hi - 1) << shift);
-    sm.remaining = remaining - excl - (first ? 0u : v0);
+    tb.prefix = prefix | ((uint32_t)(first ? d_hi : d_hi - 1) << shift);
+    tb.remaining = remaining - excl - (first ? 0u : v0);
+    tb.own_count = first ? local[0] : local[1];
   }
   __syncthreads();
 }
+
+// Block-wide exclusive prefix, in thread order, of `mine` (entries above the threshold in the low half, equal to
+// it in the high half; a CTA holds at most 16k keys).  *total: the block's sum.  One block barrier.
+__device__ __forceinline__ uint32_t packed_prefix(TopkTables& tb, uint32_t mine, int lane, int warp, uint32_t* total) {
+  uint32_t incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) tb.cnt_gt[warp] = incl;
+  __syncthreads();
+  const uint32_t ws = tb.cnt_gt[lane];
+  uint32_t before = lane < warp ? ws : 0u, all = ws;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    all += __shfl_xor_sync(0xffffffffu, all, o);
+  }
+  *total = all;
+  return before + incl - mine;
+}
+
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kTopkThreads)
 topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32_t* __restrict__ idx,
                    int64_t idx_stride, const __grid_constant__ SeqTable t, int cache_keys) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(smem_raw);
+  TopkTables& tb = sm.tb;
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TopkSmem));   // [cache_keys]
 
   pdl_trigger();
@@ -132,9 +171,9 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
   }
 
   const bool cached = slice <= cache_keys;
-  for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&sm.merged[0][0])[d] = 0u;
-  for (int d = tid; d < kBins; d += kTopkThreads) sm.hist[d] = 0u;
-  if (tid == 0) { sm.prefix = 0u; sm.remaining = (uint32_t)K; sm.n_cand = 0u; }
+  for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&tb.merged[0][0])[d] = 0u;
+  for (int d = tid; d < kBins; d += kTopkThreads) tb.hist[d] = 0u;
+  if (tid == 0) { tb.prefix = 0u; tb.remaining = (uint32_t)K; tb.n_cand = 0u; }
   if (cached) {
     for (int j = tid; j < n_own; j += kTopkThreads) keys[j] = order_key(x[j0 + j]);
   }
@@ -142,45 +181,40 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
 
   uint32_t* peer_merged[kCluster];
 #pragma unroll
-  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&sm.merged[0][0], p < n_cta ? p : 0);
+  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&tb.merged[0][0], p < n_cta ? p : 0);
   bool listed = false;               // the later passes read the candidate list instead of the slice
 
   for (int pass = 0; pass < 3; ++pass) {
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
     const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
     const uint32_t hi_mask = pass == 0 ? 0u : (pass == 1 ? 0xffe00000u : 0xfffffc00u);
-    const uint32_t prefix = sm.prefix;
-    const int n_scan = listed ? (int)sm.n_cand : n_own;
+    const uint32_t prefix = tb.prefix;
+    const int n_scan = listed ? (int)tb.n_cand : n_own;
     for (int j = tid; j < n_scan; j += kTopkThreads) {
       const uint32_t key = listed ? sm.cand[j] : (cached ? keys[j] : order_key(x[j0 + j]));
-      if ((key & hi_mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & digit_mask], 1u);
+      if ((key & hi_mask) == prefix) atomicAdd(&tb.hist[(key >> shift) & digit_mask], 1u);
     }
     __syncthreads();
-    uint32_t local_bins[kBins / kTopkThreads];
-    push_bins(sm, peer_merged, n_cta, pass, tid, local_bins);
+    uint32_t local[2];
+    push_bins(tb, peer_merged, n_cta, pass, tid, local);
     cluster.sync();
-    select_digit(sm, pass, shift, prefix, tid, lane, warp);
+    select_digit(tb, tb.merged[pass], shift, prefix, local, tid, lane, warp);
     if (pass == 0) {
-      // keep only this CTA's keys of the selected bin, if they fit the list (their number is
-      // this CTA's own count of that bin, which the owner of the bin still holds)
-      const uint32_t digit0 = sm.prefix >> 21;
-#pragma unroll
-      for (int e = 0; e < kBins / kTopkThreads; ++e)
-        if ((uint32_t)(tid + e * kTopkThreads) == digit0) sm.list_ok = local_bins[e] <= (uint32_t)kMaxCand;
-      __syncthreads();
-      listed = sm.list_ok != 0u;           // (a flag of its own: n_cand starts to move as soon as the first thread lists)
+      // keep only this CTA's keys of the selected bin, if they fit the list
+      const uint32_t digit0 = tb.prefix >> 21;
+      listed = tb.own_count <= (uint32_t)kMaxCand;
       if (listed) {
         for (int j = tid; j < n_own; j += kTopkThreads) {
           const uint32_t key = cached ? keys[j] : order_key(x[j0 + j]);
-          if ((key >> 21) == digit0) sm.cand[atomicAdd(&sm.n_cand, 1u)] = key;
+          if ((key >> 21) == digit0) sm.cand[atomicAdd(&tb.n_cand, 1u)] = key;
         }
       }
       __syncthreads();
     }
   }
 
-  const uint32_t thr = sm.prefix;          // key of the K-th largest score
-  const uint32_t n_ties = sm.remaining;    // entries equal to it that are kept (lowest positions)
+  const uint32_t thr = tb.prefix;          // key of the K-th largest score
+  const uint32_t n_ties = tb.remaining;    // entries equal to it that are kept (lowest positions)
 
   // ordered compaction: within the CTA, warp w owns the contiguous span [w * span, (w+1) * span)
   const int span = (((n_own + kWarps - 1) / kWarps) + 31) & ~31;
@@ -191,24 +225,24 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
     n_gt += __popc(__ballot_sync(0xffffffffu, j < s1 && key > thr));
     n_eq += __popc(__ballot_sync(0xffffffffu, j < s1 && key == thr));
   }
-  if (lane == 0) { sm.cnt_gt[warp] = n_gt; sm.cnt_eq[warp] = n_eq; }
+  if (lane == 0) { tb.cnt_gt[warp] = n_gt; tb.cnt_eq[warp] = n_eq; }
   __syncthreads();
   if (warp == 0) {
-    uint32_t g = sm.cnt_gt[lane], e = sm.cnt_eq[lane];
+    uint32_t g = tb.cnt_gt[lane], e = tb.cnt_eq[lane];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       g += __shfl_xor_sync(0xffffffffu, g, o);
       e += __shfl_xor_sync(0xffffffffu, e, o);
     }
     if (lane < n_cta) {                                    // lane p tells CTA p this CTA's totals
-      *cluster.map_shared_rank(&sm.peer_gt[rank], lane) = g;
-      *cluster.map_shared_rank(&sm.peer_eq[rank], lane) = e;
+      *cluster.map_shared_rank(&tb.peer_gt[rank], lane) = g;
+      *cluster.map_shared_rank(&tb.peer_eq[rank], lane) = e;
     }
   }
   cluster.sync();                    // the last remote access of the kernel is behind every CTA
   uint32_t gt_before = 0u, eq_before = 0u;
-  for (int r = 0; r < rank; ++r) { gt_before += sm.peer_gt[r]; eq_before += sm.peer_eq[r]; }
-  for (int w = 0; w < warp; ++w) { gt_before += sm.cnt_gt[w]; eq_before += sm.cnt_eq[w]; }
+  for (int r = 0; r < rank; ++r) { gt_before += tb.peer_gt[r]; eq_before += tb.peer_eq[r]; }
+  for (int w = 0; w < warp; ++w) { gt_before += tb.cnt_gt[w]; eq_before += tb.cnt_eq[w]; }
   uint32_t pos = gt_before + min(eq_before, n_ties);
   const uint32_t lt_mask = (1u << lane) - 1u;
   for (int j = s0 + lane; j < s0 + span; j += 32) {
@@ -224,20 +258,25 @@ topk_select_kernel(const float* __restrict__ scores, int64_t score_stride, int32
   }
 }
 
-// The same selection for slices of up to 16k keys per CTA (sequences of up to 128k keys): thread t of CTA r owns the
-// kKpt CONSECUTIVE keys from position (r * 1024 + t) * kKpt and holds them in registers, so every scan is an
-// unrolled register loop, and the final order (ascending position) is the thread order: one block-wide prefix
-// sum of the threads' counts places every kept entry, no per-key ballots.  The first cluster barrier is split:
-// a CTA arrives once its tables are clear and waits only before its first remote add.
+// The same selection for slices of up to 16k keys per CTA (sequences of up to 128k keys).  Thread t of CTA r owns
+// the kKpt CONSECUTIVE keys from position (r * 1024 + t) * kKpt and holds them in registers: every scan is an
+// unrolled register loop, and the final order (ascending position) is the thread order, so one block-wide prefix
+// sum of the threads' counts places every kept entry.  Everything that does not depend on the scores (tables,
+// the first cluster barrier's arrival) runs before the wait for the kernel that writes them.  After the first
+// pass every CTA sends its candidates (the keys of the selected bin) and its count of the keys above that bin to
+// ALL CTAs of the cluster; if every CTA's candidates fit their region, each CTA finishes the selection by itself
+// on its copy of the candidates and derives the other CTAs' totals from them: two cluster barriers in all, none
+// after the exchange, so no CTA waits for another at the end.  Otherwise (a bin that holds thousands of a CTA's
+// keys) the later passes merge histograms across the cluster like the general kernel.
 template <int kKpt>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_select_reg_kernel(const float* __restrict__ scores, int64_t score_stride, int32_t* __restrict__ idx,
                        int64_t idx_stride, const __grid_constant__ SeqTable t) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  TopkSmem& sm = *reinterpret_cast<TopkSmem*>(smem_raw);
+  TopkRegSmem& sm = *reinterpret_cast<TopkRegSmem*>(smem_raw);
+  TopkTables& tb = sm.tb;
 
   pdl_trigger();
-  pdl_wait();
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int n_cta = (int)cluster.num_blocks();
@@ -247,19 +286,28 @@ topk_select_reg_kernel(const float* __restrict__ scores, int64_t score_stride, i
   const int K = t.cu_keep[b + 1] - t.cu_keep[b];
   const float* x = scores + (int64_t)kvh * score_stride + t.cu_prompt[b];
   int32_t* out = idx + (int64_t)kvh * idx_stride + t.cu_keep[b];
-
   const int base = (rank * kTopkThreads + tid) * kKpt;          // position of this thread's first key
   const int nv = max(0, min(kKpt, L - base));                   // how many of its keys exist
+
+  for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&tb.merged[0][0])[d] = 0u;
+  for (int d = tid; d < kBins; d += kTopkThreads) tb.hist[d] = 0u;
+  if (tid == 0) { tb.prefix = 0u; tb.remaining = (uint32_t)K; tb.n_cand = 0u; sm.hi_own = 0u; }
+  uint32_t* peer_merged[kCluster];
+  uint32_t* peer_cand[kCluster];
+#pragma unroll
+  for (int p = 0; p < kCluster; ++p) {
+    peer_merged[p] = cluster.map_shared_rank(&tb.merged[0][0], p < n_cta ? p : 0);
+    peer_cand[p] = cluster.map_shared_rank(&sm.cand[0][0], p < n_cta ? p : 0);
+  }
+  __syncthreads();
+  cluster_arrive();                  // this CTA runs and its tables are clear
+  pdl_wait();                        // the scores are written, and the index buffer's last reader is done
+
   if (K >= L) {                      // keep everything (uniform over the cluster)
+    cluster_wait();
     for (int e = 0; e < nv; ++e) out[base + e] = base + e;
     return;
   }
-
-  for (int d = tid; d < 3 * kBins; d += kTopkThreads) (&sm.merged[0][0])[d] = 0u;
-  for (int d = tid; d < kBins; d += kTopkThreads) sm.hist[d] = 0u;
-  if (tid == 0) { sm.prefix = 0u; sm.remaining = (uint32_t)K; sm.n_cand = 0u; }
-  __syncthreads();
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // this CTA runs and its tables are clear
 
   uint32_t key[kKpt];
   const float* xp = x + base;
@@ -275,89 +323,116 @@ topk_select_reg_kernel(const float* __restrict__ scores, int64_t score_stride, i
   }
 #pragma unroll
   for (int e = 0; e < kKpt; ++e)
-    if (e < nv) atomicAdd(&sm.hist[key[e] >> 21], 1u);
+    if (e < nv) atomicAdd(&tb.hist[key[e] >> 21], 1u);
   __syncthreads();
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");     // every CTA of the cluster has done so
+  cluster_wait();                    // every CTA of the cluster has arrived: remote adds may start
 
-  uint32_t* peer_merged[kCluster];
-#pragma unroll
-  for (int p = 0; p < kCluster; ++p) peer_merged[p] = cluster.map_shared_rank(&sm.merged[0][0], p < n_cta ? p : 0);
-  bool listed = false;
+  uint32_t local[2];
+  push_bins(tb, peer_merged, n_cta, 0, tid, local);
+  cluster.sync();
+  select_digit(tb, tb.merged[0], 21, 0u, local, tid, lane, warp);
 
-  for (int pass = 0; pass < 3; ++pass) {
-    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-    const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
-    const uint32_t hi_mask = pass == 1 ? 0xffe00000u : 0xfffffc00u;
-    const uint32_t prefix = sm.prefix;
-    if (pass > 0) {
-      if (listed) {
-        const int n_cand = (int)sm.n_cand;
-        for (int j = tid; j < n_cand; j += kTopkThreads) {
-          const uint32_t c = sm.cand[j];
-          if ((c & hi_mask) == prefix) atomicAdd(&sm.hist[(c >> shift) & digit_mask], 1u);
-        }
-      } else {
+  // exchange: candidates and the count of the keys above the selected bin, to every CTA of the cluster
+  const uint32_t prefix0 = tb.prefix, digit0 = prefix0 >> 21;
+  const uint32_t own = tb.own_count;
+  const bool fits = own <= (uint32_t)kRegion;
+  uint32_t hi = 0u;
 #pragma unroll
-        for (int e = 0; e < kKpt; ++e)
-          if (e < nv && (key[e] & hi_mask) == prefix) atomicAdd(&sm.hist[(key[e] >> shift) & digit_mask], 1u);
-      }
-      __syncthreads();
+  for (int e = 0; e < kKpt; ++e) {
+    if (e < nv) {
+      const uint32_t d = key[e] >> 21;
+      hi += d > digit0 ? 1u : 0u;
+      if (d == digit0 && fits) sm.cand[rank][atomicAdd(&tb.n_cand, 1u)] = key[e];
     }
-    uint32_t local_bins[kBins / kTopkThreads];
-    push_bins(sm, peer_merged, n_cta, pass, tid, local_bins);
-    cluster.sync();
-    select_digit(sm, pass, shift, prefix, tid, lane, warp);
-    if (pass == 0) {
-      const uint32_t digit0 = sm.prefix >> 21;
+  }
 #pragma unroll
-      for (int e = 0; e < kBins / kTopkThreads; ++e)
-        if ((uint32_t)(tid + e * kTopkThreads) == digit0) sm.list_ok = local_bins[e] <= (uint32_t)kMaxCand;
-      __syncthreads();
-      listed = sm.list_ok != 0u;
-      if (listed) {
+  for (int o = 16; o > 0; o >>= 1) hi += __shfl_xor_sync(0xffffffffu, hi, o);
+  if (lane == 0 && hi) atomicAdd(&sm.hi_own, hi);
+  __syncthreads();
+  if (fits) {
+    for (int j = tid; j < (int)own; j += kTopkThreads) {
+      const uint32_t c = sm.cand[rank][j];
 #pragma unroll
-        for (int e = 0; e < kKpt; ++e)
-          if (e < nv && (key[e] >> 21) == digit0) sm.cand[atomicAdd(&sm.n_cand, 1u)] = key[e];
+      for (int p = 0; p < kCluster; ++p)
+        if (p < n_cta && p != rank) peer_cand[p][rank * kRegion + j] = c;
+    }
+  }
+  if (tid < n_cta) {
+    *cluster.map_shared_rank(&sm.peer_cnt[rank], tid) = own;
+    *cluster.map_shared_rank(&sm.peer_hi[rank], tid) = sm.hi_own;
+  }
+  cluster.sync();
+  bool all_fit = true;               // the same eight counts in every CTA: the whole cluster takes one branch
+  for (int r = 0; r < n_cta; ++r) all_fit = all_fit && sm.peer_cnt[r] <= (uint32_t)kRegion;
+
+  uint32_t gt_before = 0u, eq_before = 0u;   // of the CTAs before this one
+  if (all_fit) {
+    // passes 2 and 3 on this CTA's copy of all candidates (tables 1 and 2 serve as local histograms)
+    for (int pass = 1; pass < 3; ++pass) {
+      const int shift = pass == 1 ? 10 : 0;
+      const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
+      const uint32_t hi_mask = pass == 1 ? 0xffe00000u : 0xfffffc00u;
+      const uint32_t prefix = tb.prefix;
+      {                              // warps w, w + n_cta, ... share the candidates of CTA w % n_cta
+        const int r = warp % n_cta, n = (int)sm.peer_cnt[r];
+        for (int j = (warp / n_cta) * 32 + lane; j < n; j += 32 * (kWarps / n_cta)) {
+          const uint32_t c = sm.cand[r][j];
+          if ((c & hi_mask) == prefix) atomicAdd(&tb.merged[pass][(c >> shift) & digit_mask], 1u);
+        }
       }
       __syncthreads();
+      select_digit(tb, tb.merged[pass], shift, prefix, local, tid, lane, warp);
+    }
+    const uint32_t thr = tb.prefix;
+    if (warp < n_cta) {              // warp r: the totals of CTA r
+      const int n = (int)sm.peer_cnt[warp];
+      uint32_t g = 0u, q = 0u;
+      for (int j = lane; j < n; j += 32) {
+        const uint32_t c = sm.cand[warp][j];
+        g += c > thr ? 1u : 0u;
+        q += c == thr ? 1u : 0u;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        g += __shfl_xor_sync(0xffffffffu, g, o);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+      }
+      if (lane == 0) { sm.reg_gt[warp] = g + sm.peer_hi[warp]; sm.reg_eq[warp] = q; }
+    }
+  } else {
+    for (int pass = 1; pass < 3; ++pass) {
+      const int shift = pass == 1 ? 10 : 0;
+      const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
+      const uint32_t hi_mask = pass == 1 ? 0xffe00000u : 0xfffffc00u;
+      const uint32_t prefix = tb.prefix;
+#pragma unroll
+      for (int e = 0; e < kKpt; ++e)
+        if (e < nv && (key[e] & hi_mask) == prefix) atomicAdd(&tb.hist[(key[e] >> shift) & digit_mask], 1u);
+      __syncthreads();
+      push_bins(tb, peer_merged, n_cta, pass, tid, local);
+      cluster.sync();
+      select_digit(tb, tb.merged[pass], shift, prefix, local, tid, lane, warp);
     }
   }
 
-  const uint32_t thr = sm.prefix;          // key of the K-th largest score
-  const uint32_t n_ties = sm.remaining;    // entries equal to it that are kept (lowest positions)
-
-  // per thread: entries above the threshold (low half) and equal to it (high half; a CTA holds at most 16k keys)
+  const uint32_t thr = tb.prefix;          // key of the K-th largest score
+  const uint32_t n_ties = tb.remaining;    // entries equal to it that are kept (lowest positions)
   uint32_t mine = 0u;
 #pragma unroll
   for (int e = 0; e < kKpt; ++e)
     if (e < nv) mine += (key[e] > thr ? 1u : 0u) + (key[e] == thr ? 0x10000u : 0u);
-  uint32_t incl = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  if (lane == 31) sm.cnt_gt[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const uint32_t ws = sm.cnt_gt[lane];
-    uint32_t wi = ws;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
+  uint32_t total;
+  const uint32_t before = packed_prefix(tb, mine, lane, warp, &total);   // (its barrier also publishes reg_gt / reg_eq)
+  if (all_fit) {
+    for (int r = 0; r < rank; ++r) { gt_before += sm.reg_gt[r]; eq_before += sm.reg_eq[r]; }
+  } else {
+    if (tid < n_cta) {                                     // thread p tells CTA p this CTA's totals
+      *cluster.map_shared_rank(&tb.peer_gt[rank], tid) = total & 0xffffu;
+      *cluster.map_shared_rank(&tb.peer_eq[rank], tid) = total >> 16;
     }
-    sm.cnt_eq[lane] = wi - ws;                             // packed counts of the warps before this one
-    const uint32_t total = __shfl_sync(0xffffffffu, wi, 31);
-    if (lane < n_cta) {                                    // lane p tells CTA p this CTA's totals
-      *cluster.map_shared_rank(&sm.peer_gt[rank], lane) = total & 0xffffu;
-      *cluster.map_shared_rank(&sm.peer_eq[rank], lane) = total >> 16;
-    }
+    cluster.sync();                  // the last remote access of the kernel is behind every CTA
+    for (int r = 0; r < rank; ++r) { gt_before += tb.peer_gt[r]; eq_before += tb.peer_eq[r]; }
   }
-  cluster.sync();                    // the last remote access of the kernel is behind every CTA
-  uint32_t gt_before = 0u, eq_before = 0u;
-  for (int r = 0; r < rank; ++r) { gt_before += sm.peer_gt[r]; eq_before += sm.peer_eq[r]; }
-  const uint32_t before = sm.cnt_eq[warp] + (incl - mine);
   gt_before += before & 0xffffu;
   eq_before += before >> 16;
   uint32_t pos = gt_before + min(eq_before, n_ties);
@@ -385,10 +460,10 @@ cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx,
   cudaError_t e;
   if (slice <= 16 * kTopkThreads) {                                   // keys in registers: 4, 8 or 16 per thread
     auto launch = [&](auto kernel) {
-      cudaError_t le = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TopkSmem));
+      cudaError_t le = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TopkRegSmem));
       if (le != cudaSuccess) return le;
       log->begin(kKindTopk, s);
-      le = launch_pdl(kernel, grid, block, sizeof(TopkSmem), s, n_cta, scores, score_stride, idx, idx_stride, t);
+      le = launch_pdl(kernel, grid, block, sizeof(TopkRegSmem), s, n_cta, scores, score_stride, idx, idx_stride, t);
       log->end(s);
       return le != cudaSuccess ? le : cudaGetLastError();
     };

@@ -206,6 +206,47 @@ def test_topk_exact_with_ties(dq, lens, keep):
     dq.dapq_destroy(ctx)
 
 
+@pytest.mark.parametrize("case", ["heavy_tail_128k", "heavy_tail_batch", "half_constant", "signed", "two_level"])
+def test_topk_score_distributions(dq, case):
+    """Score distributions that drive the selection through its different routes: few candidates in the
+    threshold's bin (each CTA finishes on its copy of the cluster's candidates), a bin that holds thousands of
+    one CTA's keys but few of another's (the cluster falls back to merged histograms), aligned and unaligned
+    starts, negative scores."""
+    rng = np.random.default_rng(11)
+    if case == "heavy_tail_128k":
+        lens, keep = (131072,), (3932,)
+        s = rng.lognormal(0.0, 1.5, size=(2, sum(lens))).astype(np.float32)
+    elif case == "heavy_tail_batch":
+        lens, keep = (32768, 32768, 1000, 20001), (983, 100, 999, 600)
+        s = rng.lognormal(-9.0, 1.0, size=(2, sum(lens))).astype(np.float32)
+        s[1, 40000:40200] = s[1, 39999]                  # a run of ties that straddles the threshold or not
+    elif case == "half_constant":
+        lens, keep = (65536,), (40000,)
+        s = rng.uniform(0.0, 2.0, size=(2, sum(lens))).astype(np.float32)
+        s[0, :32768] = 1.0                               # the threshold falls inside 32768 equal scores
+        s[1, 1::2] = 1.0
+    elif case == "signed":
+        lens, keep = (50000, 7), (25000, 3)
+        s = rng.standard_normal((2, sum(lens))).astype(np.float32)
+        s[1] = np.round(s[1] * 4) / 4 + 0.0              # ties on both sides of zero (no negative zeros)
+        s[s == 0] = 0.0
+    else:
+        lens, keep = (100000,), (5000,)
+        s = np.where(rng.random((2, sum(lens))) < 0.04, 3.0, 1.0).astype(np.float32)   # two values only
+        s[1] += (rng.random(sum(lens)) < 0.5) * np.float32(2 ** -22)                   # ... and a last-bit split
+    w = _small(lens=lens, keep=keep, n_q_heads=2, n_kv_heads=2, n_pseudo=4, n_needles=0, outlier_channels=0)
+    ctx = _ctx(dq, w)
+    idx = torch.full((2, int(w.cu_keep[-1])), -1, dtype=torch.int32, device="cuda")
+    dq.dapq_topk_select(ctx, torch.from_numpy(s).cuda(), w.cu_prompt, keep, idx)
+    torch.cuda.synchronize()
+    got = idx.cpu().numpy()
+    for b in range(len(lens)):
+        for h in range(2):
+            ref = orc.topk_select(s[h, w.cu_prompt[b]:w.cu_prompt[b + 1]].astype(np.float64), keep[b])
+            np.testing.assert_array_equal(got[h, w.cu_keep[b]:w.cu_keep[b + 1]], ref, err_msg=f"{case} b={b} h={h}")
+    dq.dapq_destroy(ctx)
+
+
 # --------------------------------------------------------------------------- dapq_compact_kv
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_compact_bit_exact_given_oracle_indices(dq, dtype):
