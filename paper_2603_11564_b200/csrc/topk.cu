@@ -13,7 +13,7 @@
 // entry.  No CTA ever reads remote memory, and none has to outlive another.
 //   topk_select_reg_kernel (slices of up to 32k keys: sequences of up to 256k keys): keys in registers; after the
 //     first pass the CTAs exchange the keys of the selected bin and finish by themselves (see the kernel).
-//   topk_select_solo_kernel: the same with one CTA per head (batches of sequences of up to 32k keys).
+//   topk_select_solo_kernel: the same with one CTA per head (short sequences, batches of sequences of up to 16k keys).
 //   topk_select_kernel (longer slices): keys in shared memory or re-read from global memory; every pass merges
 //     histograms across the cluster, and the CTAs push their totals to each other before the ordered write.
 #include <cooperative_groups.h>
@@ -455,7 +455,7 @@ topk_select_reg_kernel(const float* __restrict__ scores, int64_t score_stride, i
   }
 }
 
-// One CTA per (sequence, KV head), for sequences of up to 32k keys when a cluster per head would not fit one wave
+// One CTA per (sequence, KV head), for sequences of up to 16k keys when a cluster per head would not fit one wave
 // (batches): the same steps as topk_select_reg_kernel without any exchange: the three tables are local histograms.
 template <int kKpt>
 __global__ void __launch_bounds__(kTopkThreads)
@@ -504,10 +504,11 @@ topk_select_solo_kernel(const float* __restrict__ scores, int64_t score_stride, 
   const uint32_t local[2] = {0u, 0u};
   select_digit(tb, tb.merged[0], 21, 0u, local, tid, lane, warp);
 
+  // the selected bin's keys (the candidates) go to the list (a CTA's keys always fit it); the later passes read it
+  static_assert(kKpt * kTopkThreads <= kCap, "one CTA's keys must fit the candidate list");
   const uint32_t digit0 = tb.prefix >> 21;
   const int n_all = (int)tb.bin_total;
-  const bool listed = n_all <= kCap;         // the selected bin's keys fit the list: the later passes read it
-  if (listed) {
+  {
     uint32_t mine = 0u;
 #pragma unroll
     for (int e = 0; e < kKpt; ++e)
@@ -531,15 +532,9 @@ topk_select_solo_kernel(const float* __restrict__ scores, int64_t score_stride, 
     const uint32_t digit_mask = pass == 2 ? 1023u : 2047u;
     const uint32_t hi_mask = pass == 1 ? 0xffe00000u : 0xfffffc00u;
     const uint32_t prefix = tb.prefix;
-    if (listed) {
-      for (int j = tid; j < n_all; j += kTopkThreads) {
-        const uint32_t c = sm.cand[j];
-        if ((c & hi_mask) == prefix) atomicAdd(&tb.merged[pass][(c >> shift) & digit_mask], 1u);
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < kKpt; ++e)
-        if (e < nv && (key[e] & hi_mask) == prefix) atomicAdd(&tb.merged[pass][(key[e] >> shift) & digit_mask], 1u);
+    for (int j = tid; j < n_all; j += kTopkThreads) {
+      const uint32_t c = sm.cand[j];
+      if ((c & hi_mask) == prefix) atomicAdd(&tb.merged[pass][(c >> shift) & digit_mask], 1u);
     }
     __syncthreads();
     select_digit(tb, tb.merged[pass], shift, prefix, local, tid, lane, warp);
@@ -582,6 +577,7 @@ TopkShape plan_topk(int heads, int max_len, int n_sm) {
     const int slice = (max_len + n_cta - 1) / n_cta;
     if (slice > 32 * kTopkThreads) continue;
     const int kpt = slice <= 4 * kTopkThreads ? 4 : (slice <= 8 * kTopkThreads ? 8 : (slice <= 16 * kTopkThreads ? 16 : 32));
+    if (n_cta == 1 && kpt == 32) continue;              // (a cluster of two with 16 keys per thread is never slower)
     const int ctas = heads * n_cta;
     const int per_sm = (kpt <= 16 && ctas > n_sm) ? 2 : 1;
     const int waves = (ctas + n_sm * per_sm - 1) / (n_sm * per_sm);
@@ -618,8 +614,7 @@ cudaError_t launch_topk(const float* scores, int64_t score_stride, int32_t* idx,
       switch (shape.kpt) {
         case 4: return launch(topk_select_solo_kernel<4>);
         case 8: return launch(topk_select_solo_kernel<8>);
-        case 16: return launch(topk_select_solo_kernel<16>);
-        default: return launch(topk_select_solo_kernel<32>);
+        default: return launch(topk_select_solo_kernel<16>);
       }
     }
     switch (shape.kpt) {

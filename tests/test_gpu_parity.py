@@ -180,6 +180,7 @@ def test_score_strided_view_and_custom_scale(dq):
 @pytest.mark.parametrize("lens,keep", [
     ((1, 33, 4096, 5000, 131072, 77), (1, 33, 1, 4999, 3932, 200)),
     ((400000, 9), (12345, 3)),       # slices too long for the shared-memory key cache
+    ((200000, 130000), (7000, 129999)),   # 32 keys per thread
 ])
 def test_topk_exact_with_ties(dq, lens, keep):
     rng = np.random.default_rng(5)
@@ -206,7 +207,7 @@ def test_topk_exact_with_ties(dq, lens, keep):
     dq.dapq_destroy(ctx)
 
 
-@pytest.mark.parametrize("case", ["heavy_tail_128k", "heavy_tail_batch", "half_constant", "signed", "two_level"])
+@pytest.mark.parametrize("case", ["heavy_tail_128k", "heavy_tail_batch", "half_constant", "signed", "two_level", "many_heads"])
 def test_topk_score_distributions(dq, case):
     """Score distributions that drive the selection through its different routes: few candidates in the
     threshold's bin (each CTA finishes on its copy of the cluster's candidates), a bin that holds thousands of
@@ -230,18 +231,24 @@ def test_topk_score_distributions(dq, case):
         s = rng.standard_normal((2, sum(lens))).astype(np.float32)
         s[1] = np.round(s[1] * 4) / 4 + 0.0              # ties on both sides of zero (no negative zeros)
         s[s == 0] = 0.0
-    else:
+    elif case == "two_level":
         lens, keep = (100000,), (5000,)
         s = np.where(rng.random((2, sum(lens))) < 0.04, 3.0, 1.0).astype(np.float32)   # two values only
         s[1] += (rng.random(sum(lens)) < 0.5) * np.float32(2 ** -22)                   # ... and a last-bit split
-    w = _small(lens=lens, keep=keep, n_q_heads=2, n_kv_heads=2, n_pseudo=4, n_needles=0, outlier_channels=0)
+    else:                                                # 320 heads of 12k keys: one CTA per head, two per SM
+        lens, keep = (12000,) * 20, tuple(range(100, 2100, 100))
+        s = rng.lognormal(0.0, 0.5, size=(16, sum(lens))).astype(np.float32)
+        s[3] = np.round(s[3] * 8) / 8
+        s[5] = 1.0
+    H = s.shape[0]
+    w = _small(lens=lens, keep=keep, n_q_heads=H, n_kv_heads=H, n_pseudo=4, n_needles=0, outlier_channels=0)
     ctx = _ctx(dq, w)
-    idx = torch.full((2, int(w.cu_keep[-1])), -1, dtype=torch.int32, device="cuda")
+    idx = torch.full((H, int(w.cu_keep[-1])), -1, dtype=torch.int32, device="cuda")
     dq.dapq_topk_select(ctx, torch.from_numpy(s).cuda(), w.cu_prompt, keep, idx)
     torch.cuda.synchronize()
     got = idx.cpu().numpy()
     for b in range(len(lens)):
-        for h in range(2):
+        for h in range(H):
             ref = orc.topk_select(s[h, w.cu_prompt[b]:w.cu_prompt[b + 1]].astype(np.float64), keep[b])
             np.testing.assert_array_equal(got[h, w.cu_keep[b]:w.cu_keep[b + 1]], ref, err_msg=f"{case} b={b} h={h}")
     dq.dapq_destroy(ctx)
