@@ -181,6 +181,7 @@ struct QgPlan {
   CUtensorMap tm_k1, tm_k2, tm_q;
   ChunkTable ct1, ct2;
   int32_t n_qgroups, rows_g, n_stages1, n_stages2, q_is_f16;
+  int32_t n_qgroups2, rows_g2, wide2;     // sweep 2's own cut of the query rows (groups of up to 512 rows when wide2)
 };
 int qg_groups(const Dims& dm);
 bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t, const Dims& dm, int n_sm, QgPlan* plan);

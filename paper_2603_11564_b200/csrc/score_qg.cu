@@ -145,14 +145,22 @@ bool qg_plan(const void* q, int q_is_f16, const CacheDev& cv, const SeqTable& t,
   plan->q_is_f16 = q_is_f16;
   const int q_bytes = ((plan->rows_g + 127) / 128) * 2 * 128 * 128;
   const int s1 = (kRingEnd - (q_is_f16 ? kRefSlabBytes : 0) - q_bytes) / TileGeo<kTile1>::kStage;   // (the reference operand sits at the end)
-  const int s2 = (kRingEnd - (q_is_f16 ? kSlabBytes : 0) - q_bytes) / TileGeo<kTile2>::kStage;   // (the -lse operands sit at the end)
   plan->n_stages1 = s1 < kMaxStages ? s1 : kMaxStages;
+  // Sweep 2 keeps up to 512 query rows per CTA when a KV head has more than 256 (two jobs per K tile): half as
+  // many CTAs fetch and convert every tile, and half as many score slots are written.
+  plan->wide2 = rows_total > kGroupRows ? 1 : 0;
+  plan->n_qgroups2 = plan->wide2 ? (rows_total + kWideRows - 1) / kWideRows : plan->n_qgroups;
+  plan->rows_g2 = plan->wide2 ? (((rows_total + plan->n_qgroups2 - 1) / plan->n_qgroups2) + 15) & ~15 : plan->rows_g;
+  const int q_bytes2 = ((plan->rows_g2 + 127) / 128) * 2 * 128 * 128;
+  const int ring2 = plan->wide2 ? SmemT<true>::ring_end - (q_is_f16 ? SmemT<true>::slab_bytes : 0)
+                                : kRingEnd - (q_is_f16 ? kSlabBytes : 0);                          // (the -lse operands sit at the end)
+  const int s2 = (ring2 - q_bytes2) / TileGeo<kTile2>::kStage;
   plan->n_stages2 = s2 < kMaxStages ? s2 : kMaxStages;
-  const int ctas = dm.n_kv_heads * plan->n_qgroups;
+  if (plan->n_stages1 < 2 || plan->n_stages2 < 2) return false;
   // (a sweep-2 tile is one job of about a microsecond, a sweep-1 tile two: a CTA's set-up of several
   // microseconds weighs more tiles in sweep 2, where ragged batches would otherwise be cut into waves of short CTAs)
-  if (!plan_chunks(t, dm.n_pseudo, kTile1, ctas, n_sm, &plan->ct1, 3.0)) return false;
-  if (!plan_chunks(t, 0, kTile2, ctas, n_sm, &plan->ct2, 6.0)) return false;
+  if (!plan_chunks(t, dm.n_pseudo, kTile1, dm.n_kv_heads * plan->n_qgroups, n_sm, &plan->ct1, 3.0)) return false;
+  if (!plan_chunks(t, 0, kTile2, dm.n_kv_heads * plan->n_qgroups2, n_sm, &plan->ct2, plan->wide2 ? 3.0 : 6.0)) return false;
   // ---- tensor maps: K as [d, rows, H_kv] (one map per sweep: the boxes differ), the query operand as [d, rows]
   const uint64_t rows_k = (uint64_t)t.cu_rows[t.batch];
   const uint64_t kd[3] = {(uint64_t)kHeadDim, rows_k, (uint64_t)dm.n_kv_heads};
@@ -186,13 +194,13 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
   a.lse_out = lse_out;
   a.score_stride = score_stride;
   a.slot_stride = (int64_t)dm.n_kv_heads * score_stride;
-  a.scores = plan.n_qgroups > 1 ? slots : scores;
+  a.scores = plan.n_qgroups2 > 1 ? slots : scores;
   a.status = status;
 
-  auto run = [&](auto sweep1, auto sweep2) -> cudaError_t {
+  auto run = [&](auto sweep1, auto sweep2, int smem2) -> cudaError_t {
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(sweep1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(sweep2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(sweep2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2)) != cudaSuccess) return e;
     if (lse_in == nullptr) {
       a.n_stages = plan.n_stages1;
       a.early_loads = after_own_kernel ? 1 : 0;
@@ -202,25 +210,33 @@ cudaError_t launch_score_qg(const QgPlan& plan, const SeqTable& t, const Dims& d
       log->end(s);
       if (e != cudaSuccess) return e;
     }
+    a.n_qgroups = plan.n_qgroups2;                                       // sweep 2's own cut of the query rows
+    a.rows_g = plan.rows_g2;
     a.n_stages = plan.n_stages2;
     a.early_loads = (after_own_kernel || lse_in == nullptr) ? 1 : 0;     // (sweep 1, if it ran, waited for what came before)
     log->begin(kKindSweep2, s);
-    e = launch_pdl(sweep2, dim3(plan.ct2.n_chunks * plan.n_qgroups, dm.n_kv_heads), dim3(kThreads2), kSmemBytes, s, 1,
+    e = launch_pdl(sweep2, dim3(plan.ct2.n_chunks * plan.n_qgroups2, dm.n_kv_heads), dim3(kThreads2), smem2, s, 1,
                    plan.tm_k2, plan.tm_q, t, plan.ct2, plan.ct1, a);
     log->end(s);
     return e;
   };
-  cudaError_t e = plan.q_is_f16 ? run(rowstat_kernel<true>, colsum_kernel<true>) : run(rowstat_kernel<false>, colsum_kernel<false>);
+  cudaError_t e;
+  if (plan.wide2)
+    e = plan.q_is_f16 ? run(rowstat_kernel<true>, colsum_kernel<true, true>, SmemT<true>::total)
+                      : run(rowstat_kernel<false>, colsum_kernel<false, true>, SmemT<true>::total);
+  else
+    e = plan.q_is_f16 ? run(rowstat_kernel<true>, colsum_kernel<true, false>, kSmemBytes)
+                      : run(rowstat_kernel<false>, colsum_kernel<false, false>, kSmemBytes);
   if (e != cudaSuccess) return e;
-  if (plan.n_qgroups > 1) {
+  if (plan.n_qgroups2 > 1) {
     const int64_t count = (int64_t)dm.n_kv_heads * score_stride;
     log->begin(kKindSlotSum, s);
     if (count % 4 == 0 && a.slot_stride % 4 == 0 && ((uintptr_t)slots & 15u) == 0 && ((uintptr_t)scores & 15u) == 0)
       e = launch_pdl(score_slots_sum_kernel, dim3((unsigned)((count / 4 + 255) / 256)), dim3(256), 0, s, 1,
-                     (const float4*)slots, plan.n_qgroups, a.slot_stride / 4, (float4*)scores, count / 4);
+                     (const float4*)slots, plan.n_qgroups2, a.slot_stride / 4, (float4*)scores, count / 4);
     else
       e = launch_pdl(score_slots_sum1_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, s, 1, (const float*)slots,
-                     plan.n_qgroups, a.slot_stride, scores, count);
+                     plan.n_qgroups2, a.slot_stride, scores, count);
     log->end(s);
     if (e != cudaSuccess) return e;
   }

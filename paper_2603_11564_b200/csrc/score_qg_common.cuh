@@ -22,15 +22,12 @@ constexpr int kThreads2 = kThreads1 + 32;                               // sweep
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 4, kMaxAcc = 4;
 constexpr int kExchDepth = 4;                  // jobs whose partial sums can wait in shared memory (sweep 2)
-constexpr int kRingEnd = 216 * 1024;           // queries + K ring end here; the small state follows
+constexpr int kWideRows = 2 * kGroupRows;      // ... in the wide form of sweep 2 (two accumulators' worth of query columns)
 // Sweep 2 with its own fp16 queries appends one k-step to every job's MMAs that adds -lse_i to column i of
-// the accumulator: a [256 x 16] operand holding -lse as an fp16 pair, against a [128 x 16] operand of ones.
-constexpr int kLseSlabBytes = kGroupRows * 32, kOnesSlabBytes = kTile2 * 32;
-constexpr int kSlabBytes = kLseSlabBytes + kOnesSlabBytes;                      // kept at the end of the ring area
-constexpr int kLseSlab = kRingEnd - kSlabBytes, kOnesSlab = kRingEnd - kOnesSlabBytes;
+// the accumulator: a [rows x 16] operand holding -lse as an fp16 pair, against a [128 x 16] operand of ones.
 // Sweep 1 does the same with a per-row reference logit (its [256 x 16] operand also sits at the end of the
 // ring area; its [192 x 16] operand of ones takes the place of sweep 2's exchange ring behind the barriers).
-constexpr int kRefSlabBytes = kGroupRows * 32, kRefSlab = kRingEnd - kRefSlabBytes, kOnes1SlabBytes = kTile1 * 32;
+constexpr int kOnesSlabBytes = kTile2 * 32, kOnes1SlabBytes = kTile1 * 32;
 
 template <int kTile>
 struct TileGeo {
@@ -38,23 +35,35 @@ struct TileGeo {
   static constexpr int kHalf = kTile * 128;
 };
 
-// Shared memory behind the ring (offsets from the 1024-aligned base).
-struct Smem {
-  static constexpr int bars = kRingEnd;
+// Shared memory (offsets from the 1024-aligned base): queries, K ring and the extra operands up to ring_end,
+// the small state behind it.  kWide: room for 512 query rows (sweep 2 only).
+template <bool kWide>
+struct SmemT {
+  static constexpr int rows = kWide ? kWideRows : kGroupRows;
+  static constexpr int ring_end = (kWide ? 214 : 216) * 1024;
+  static constexpr int lse_slab_bytes = rows * 32, slab_bytes = lse_slab_bytes + kOnesSlabBytes;
+  static constexpr int lse_slab = ring_end - slab_bytes, ones_slab = ring_end - kOnesSlabBytes;   // sweep 2's extra operands
+  static constexpr int ref_slab_bytes = rows * 32, ref_slab = ring_end - ref_slab_bytes;          // sweep 1's
+  static constexpr int bars = ring_end;
   // barriers: k_full[4], k_conv[4], k_empty[4], acc_full[4], acc_empty[4], part_full[4], part_empty[4], q_full, drain, lse_ready
   static constexpr int n_bars = 3 * kMaxStages + 2 * kMaxAcc + 2 * kExchDepth + 3;
-  static constexpr int lse = (bars + n_bars * 8 + 15) & ~15;       // [256] floats, read as float4 (sweep 2); with the next block:
-                                                                   // [256] float2 row statistics (sweep 1)
-  static constexpr int aux = lse + kGroupRows * 4;                 // [256] floats: the other half of the statistics
-  static constexpr int exch = aux + kGroupRows * 4;                // [kExchDepth][4][128] floats (sweep 2)
+  static constexpr int lse = (bars + n_bars * 8 + 15) & ~15;       // [rows] floats, read as float4 (sweep 2); with the next block:
+                                                                   // [rows] float2 row statistics (sweep 1)
+  static constexpr int aux = lse + rows * 4;                       // [rows] floats: the other half of the statistics
+  static constexpr int exch = aux + rows * 4;                      // [kExchDepth][4][128] floats (sweep 2)
   static constexpr int tmem_ptr = exch + kExchDepth * kEpiGroups * 128 * 4;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
+  static_assert(lse % 16 == 0 && aux % 16 == 0 && exch % 256 == 0, "vector loads need 16-byte alignment, MMA operands 256");
+  static_assert(total <= 232448, "exceeds the shared memory a CTA can opt in to");
 };
-static_assert(Smem::lse % 16 == 0 && Smem::aux % 16 == 0 && Smem::exch % 256 == 0, "vector loads need 16-byte alignment, MMA operands 256");
+using Smem = SmemT<false>;
+constexpr int kRingEnd = Smem::ring_end;
+constexpr int kLseSlabBytes = Smem::lse_slab_bytes, kSlabBytes = Smem::slab_bytes;
+constexpr int kLseSlab = Smem::lse_slab, kOnesSlab = Smem::ones_slab;
+constexpr int kRefSlabBytes = Smem::ref_slab_bytes, kRefSlab = Smem::ref_slab;
 static_assert(kOnes1SlabBytes <= kExchDepth * kEpiGroups * 128 * 4, "sweep 1's operand of ones does not fit the exchange area");
 constexpr int kSmemBytes = Smem::total;
-static_assert(kSmemBytes <= 232448, "exceeds the shared memory a CTA can opt in to");
 
 struct Args {
   int32_t n_pseudo, group, n_q_heads, n_kv_heads;
@@ -150,7 +159,7 @@ __device__ __forceinline__ uint32_t bar_count(int idx) {
 // thread 0 as soon as the barriers exist: only copies of data that the kernel before this one does not
 // write), tensor-memory allocation (warp 1), one CTA-wide sync, then the wait for the kernel before this one
 // (all of this overlaps that kernel's tail).  Returns the tensor-memory base address.
-template <class First>
+template <class Smem = SmemT<false>, class First>
 __device__ __forceinline__ uint32_t cta_prologue(uint8_t* smem, uint32_t sbase, const Bars& bars, First first) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   static_assert(Smem::n_bars <= 32, "one barrier per lane of warp 0");

@@ -78,7 +78,10 @@ __device__ __forceinline__ float colsum_job(uint32_t taddr, const float* lse_s, 
   return (acc.x + acc.y) + (acc1.x + acc1.y);
 }
 
-template <bool kConvert>
+// kWide: the CTA keeps up to 512 query rows resident and runs two jobs per K tile (query columns 0..255 and
+// 256..); a thread adds its two jobs' sums before it posts them, so a tile is fetched, converted and stored once
+// for twice the queries.
+template <bool kConvert, bool kWide>
 __global__ void __launch_bounds__(kThreads2, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ SeqTable t, const __grid_constant__ ChunkTable ct,
@@ -96,16 +99,19 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
   const Work w = cta_work(t, ct, a, kTile2, false);
   const int nt = w.nt, L = w.L, b = w.b;
   if (nt <= 0) return;
+  using Smem = SmemT<kWide>;
   const Bars bars{sbase + Smem::bars};
   const Waiter wt{reinterpret_cast<volatile int*>(smem + Smem::abort_flag), a.status, a.wait_limit};
-  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [256] minus the base-2 lse of the resident query rows
-  float* aux = reinterpret_cast<float*>(smem + Smem::aux);      // [256] scratch of the lse merge
+  float* lse_s = reinterpret_cast<float*>(smem + Smem::lse);    // [rows] minus the base-2 lse of the resident query rows
+  float* aux = reinterpret_cast<float*>(smem + Smem::aux);      // [rows] scratch of the lse merge
   float* exch = reinterpret_cast<float*>(smem + Smem::exch);    // [kExchDepth][4][128] partial sums on their way to the summing warp
   // The epilogue threads ask for sweep 1's partials of their query row first of all, before the CTA's copies of
   // queries and keys crowd the memory system (two threads per row: thread (eg, r) takes row (eg & 1) * 128 + r and
-  // the chunks of parity eg >> 1; up to 16 partials per thread at once).
+  // the chunks of parity eg >> 1; up to 16 partials per thread at once.  kWide: one thread per row, every chunk).
   const bool is_epi = warp >= kFirstEpiWarp && warp < kFirstEpiWarp + 4 * kEpiGroups;
-  const int m_eg = (warp - kFirstEpiWarp) >> 2, m_row = (m_eg & 1) * 128 + (warp & 3) * 32 + lane;
+  const int m_eg = (warp - kFirstEpiWarp) >> 2, m_row = (kWide ? m_eg : (m_eg & 1)) * 128 + (warp & 3) * 32 + lane;
+  constexpr int m_cs = kWide ? 1 : 2;                           // chunk stride of a thread
+  const int m_c0 = kWide ? 0 : (m_eg >> 1);                     // its first chunk
   const bool m_live = is_epi && m_row < w.rows && !a.lse_in;
   const int m_nc = ct1.cu_chunk[b + 1] - ct1.cu_chunk[b];
   const int64_t m_step = (int64_t)a.n_kv_heads * a.rows_pad;
@@ -115,14 +121,16 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     pdl_wait();                                                 // (sweep 1 wrote them)
 #pragma unroll
     for (int u = 0; u < 16; ++u)
-      m_q[u] = (m_eg >> 1) + 2 * u < m_nc ? __ldg(m_p + ((m_eg >> 1) + 2 * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
+      m_q[u] = m_c0 + m_cs * u < m_nc ? __ldg(m_p + (m_c0 + m_cs * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
   }
   // (behind this library's own sweep 1 or rotation kernel, keys and queries were complete before that kernel
   // got past its wait: both go out at once)
-  const uint32_t tmem_base = cta_prologue(smem, sbase, bars, [&] {
+  const uint32_t tmem_base = cta_prologue<Smem>(smem, sbase, bars, [&] {
     if (a.early_loads) tma_first<kTile2, true>(&tm_k, &tm_q, w, a, sbase, bars, kvh);
   });
-  const int ncols = (w.rows + 15) & ~15;                        // UMMA N: only the query columns that exist
+  // UMMA N: only the query columns that exist; job 1 (kWide) holds the rows from 256 on
+  const int ncols = (min(w.rows, kGroupRows) + 15) & ~15, ncols1 = kWide ? ((max(w.rows - kGroupRows, 0) + 15) & ~15) : 0;
+  const int n_jobs = ncols1 > 0 ? 2 : 1;                        // jobs per K tile
   const int acc_cols = ncols > 128 ? 256 : 128, n_acc = kTmemCols / acc_cols;
   const uint32_t q_half = (uint32_t)w.mb * 128u * 128u;         // bytes of one 64-channel half of the query group
   const int S = a.n_stages;
@@ -138,25 +146,33 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
       bool ok = wt.wait(bars.q_full(), 0);
       if (ok && kFold) ok = wt.wait(bars.lse_ready(), 0);
       const uint32_t idesc = kConvert ? umma_idesc_f16(128, ncols) : umma_idesc(128, ncols);
+      const uint32_t idesc1 = ncols1 ? (kConvert ? umma_idesc_f16(128, ncols1) : umma_idesc(128, ncols1)) : 0u;
       const uint64_t qd = umma_desc(sbase);
-      const uint64_t ones_d = umma_desc_rows32(sbase + kOnesSlab), lse_d = umma_desc_rows32(sbase + kLseSlab);
+      const uint64_t ones_d = umma_desc_rows32(sbase + Smem::ones_slab), lse_d = umma_desc_rows32(sbase + Smem::lse_slab);
       const uint32_t ring = sbase + 2 * q_half;
       Ring rs(S), ra(n_acc);
-      for (int ti = 0; ti < nt && ok; ++ti, rs.next(), ra.next()) {
-        const int s = rs.i, buf = ra.i;
+      for (int ti = 0; ti < nt && ok; ++ti, rs.next()) {
+        const int s = rs.i;
         ok = wt.wait(kConvert ? bars.k_conv(s) : bars.k_full(s), rs.phase);
-        if (ok && ra.wrapped) ok = wt.wait(bars.acc_empty(buf), ra.phase ^ 1u);
-        if (!ok) break;
-        tc_fence_after();
         const uint64_t kd = umma_desc(ring + s * T::kStage);
-        const uint32_t d = tmem_base + buf * acc_cols;
+        for (int jb = 0; jb < n_jobs && ok; ++jb, ra.next()) {
+          const int buf = ra.i;
+          if (ra.wrapped) ok = wt.wait(bars.acc_empty(buf), ra.phase ^ 1u);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d = tmem_base + buf * acc_cols;
+          const uint64_t qj = desc_advance(qd, jb * 2 * 128 * 128);          // query rows 256 jb ..: blocks 2 jb, 2 jb + 1
+          const uint32_t id = jb ? idesc1 : idesc;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const int half = ks >> 2, kk = ks & 3;
-          umma_ss(d, desc_advance(kd, half * T::kHalf + kk * 32), desc_advance(qd, half * q_half + kk * 32), idesc, ks ? 1u : 0u);
+          for (int ks = 0; ks < 8; ++ks) {
+            const int half = ks >> 2, kk = ks & 3;
+            umma_ss(d, desc_advance(kd, half * T::kHalf + kk * 32), desc_advance(qj, half * q_half + kk * 32), id, ks ? 1u : 0u);
+          }
+          // D[key, i] += 1 * (-lse_i) (an fp16 pair against two ones)
+          if (kFold) umma_ss(d, ones_d, desc_advance(lse_d, jb * kGroupRows * 32), id, 1u);
+          tc_commit(bars.acc_full(buf));
         }
-        if (kFold) umma_ss(d, ones_d, lse_d, idesc, 1u);        // D[key, i] += 1 * (-lse_i) (an fp16 pair against two ones)
-        tc_commit(bars.acc_full(buf));
+        if (!ok) break;
         tc_commit(bars.k_empty(s));                             // the K stage is free once these MMAs retire
       }
       mma_drain(bars);
@@ -174,15 +190,15 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // partials of row (eg & 1) * 128 + r over the chunks of parity eg >> 1, all of its loads in flight at
     // once; the odd half then crosses through shared memory and the even half finishes (fixed order).
     {
-      const int row = (eg & 1) * 128 + r, grow = w.qgrp * a.rows_g + row;
+      const int row = m_row, grow = w.qgrp * a.rows_g + row;
       const bool live = row < w.rows;
       float mx = -CUDART_INF_F, z = 0.f;
       if (m_live) {
-        for (int c0 = eg >> 1; c0 < m_nc; c0 += 32) {
-          if (c0 > (eg >> 1)) {                                 // (more than 32 chunks: the next batch)
+        for (int c0 = m_c0; c0 < m_nc; c0 += 16 * m_cs) {
+          if (c0 > m_c0) {                                      // (more chunks than one batch of 16 per thread)
 #pragma unroll
             for (int u = 0; u < 16; ++u)
-              m_q[u] = c0 + 2 * u < m_nc ? __ldg(m_p + (c0 + 2 * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
+              m_q[u] = c0 + m_cs * u < m_nc ? __ldg(m_p + (c0 + m_cs * u) * m_step) : make_float2(-CUDART_INF_F, 0.f);
           }
           float m16 = m_q[0].x;
 #pragma unroll
@@ -197,16 +213,18 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
           }
         }
       }
-      if (eg >= 2) {
+      if (!kWide && eg >= 2) {
         aux[row] = mx;
         lse_s[row] = z;                                         // (the odd half's sums, until the even half has read them)
       }
       epilogue_sync();
-      if (eg < 2) {
+      if (kWide || eg < 2) {
         float l2 = 0.f;
         if (live) {
           if (a.lse_in) {
             l2 = a.lse_in[w.qrow_base + grow] * 1.4426950408889634f;
+          } else if (kWide) {
+            l2 = mx + log2f(z);
           } else {
             const float mo = aux[row], zo = lse_s[row];
             const float m = fmaxf(mx, mo);
@@ -222,39 +240,49 @@ colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
           const __half hi = __float2half_rn(-l2);
           const __half lo = __float2half_rn(live ? -l2 - __half2float(hi) : 0.f);
           const uint32_t pair = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
-          const uint32_t dst = sbase + kLseSlab + (row >> 3) * 256 + (row & 7) * 32;
+          const uint32_t dst = sbase + Smem::lse_slab + (row >> 3) * 256 + (row & 7) * 32;
           sts128(dst, make_uint4(live ? pair : 0u, 0u, 0u, 0u));
           sts128(dst + 16, make_uint4(0u, 0u, 0u, 0u));
         }
       }
       if (kFold) {
         const int tid_e = (warp - kFirstEpiWarp) * 32 + lane;   // 0 .. 511: the ones operand, 256 pieces of 16 bytes
-        if (tid_e < kOnesSlabBytes / 16) sts128(sbase + kOnesSlab + tid_e * 16, make_uint4(0x3c003c00u, 0u, 0u, 0u));
+        if (tid_e < kOnesSlabBytes / 16) sts128(sbase + Smem::ones_slab + tid_e * 16, make_uint4(0x3c003c00u, 0u, 0u, 0u));
         fence_proxy_async();                                    // the MMAs read both operands through the async proxy
       }
       epilogue_sync();
       if (warp == kFirstEpiWarp && lane == 0) mbar_arrive(bars.lse_ready());    // (the MMA issuer and the TMA producer wait for it)
     }
     // Pieces of a job (16 query columns): group g takes pieces [g nch / 4, (g + 1) nch / 4), at most four
-    const int nch = ncols >> 4;
+    const int nch = ncols >> 4, nch1 = ncols1 >> 4;
     const int p0 = (eg * nch) / kEpiGroups, np = ((eg + 1) * nch) / kEpiGroups - p0;
-    const bool full = (p0 + np) * 16 <= w.rows;                 // no column of this warp's pieces lies beyond the group
+    const int p1 = (eg * nch1) / kEpiGroups, np1 = ((eg + 1) * nch1) / kEpiGroups - p1;
+    const bool full = (p0 + np) * 16 <= min(w.rows, kGroupRows);    // no column of this warp's pieces lies beyond the group
+    const bool full1 = (p1 + np1) * 16 <= w.rows - kGroupRows;
     bool ok = true;
     Ring ra(n_acc);
-    for (int ti = 0; ti < nt && ok; ++ti, ra.next()) {
-      const int buf = ra.i;
-      ok = __all_sync(0xffffffffu, wt.wait(bars.acc_full(buf), ra.phase));
+    for (int ti = 0; ti < nt && ok; ++ti) {
+      float sum = 0.f;
+      for (int jb = 0; jb < n_jobs && ok; ++jb, ra.next()) {
+        const int buf = ra.i;
+        ok = __all_sync(0xffffffffu, wt.wait(bars.acc_full(buf), ra.phase));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = lane_addr + buf * acc_cols;
+        // the accumulator goes back to the MMA issuer as soon as this warp's last piece is in registers
+        auto release = [&] {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.acc_empty(buf));
+        };
+        if (jb == 0)
+          sum = full ? colsum_job<true, kFold>(taddr, lse_s, p0, np, min(w.rows, kGroupRows), c, release)
+                     : colsum_job<false, kFold>(taddr, lse_s, p0, np, min(w.rows, kGroupRows), c, release);
+        else
+          sum += full1 ? colsum_job<true, kFold>(taddr, lse_s + kGroupRows, p1, np1, w.rows - kGroupRows, c, release)
+                       : colsum_job<false, kFold>(taddr, lse_s + kGroupRows, p1, np1, w.rows - kGroupRows, c, release);
+      }
       if (!ok) break;
-      tc_fence_after();
-      const uint32_t taddr = lane_addr + buf * acc_cols;
-      // the accumulator goes back to the MMA issuer as soon as this warp's last piece is in registers
-      auto release = [&] {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars.acc_empty(buf));
-      };
-      const float sum = full ? colsum_job<true, kFold>(taddr, lse_s, p0, np, w.rows, c, release)
-                             : colsum_job<false, kFold>(taddr, lse_s, p0, np, w.rows, c, release);
       const int slot = ti % kExchDepth;
       if (ti >= kExchDepth) ok = __all_sync(0xffffffffu, wt.wait(bars.part_empty(slot), ((ti / kExchDepth) - 1) & 1));
       if (!ok) break;

@@ -99,6 +99,9 @@ SCORE_CASES = [
     ("bf16", 8, 1, 128, (129, 1031)),
     ("bf16", 4, 4, 100, (777,)),
     ("bf16", 8, 2, 17, (512, 1024, 300, 5)),
+    # more than 256 query rows per KV head: sweep 2 keeps up to 512 resident, the second job narrow (48 / 16 columns)
+    ("bf16", 3, 1, 100, (600, 90)),
+    ("bf16", 5, 1, 104, (700,)),
     # CUDA-core sweeps at every chunk size (512 / 256 / 128 keys on a 148-SM part; the shorter cases above take 64)
     ("f32", 8, 8, 8, (19000,)),
     ("bf16", 8, 8, 4, (9000, 700)),
