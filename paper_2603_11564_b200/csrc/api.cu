@@ -28,7 +28,7 @@ struct dapq_ctx {
   float* lse2 = nullptr;         // [max_batch, H_q, N]
   float* scores = nullptr;       // [H_kv, max_total_rows]
   float* pooled = nullptr;       // [H_kv, max_total_rows] (pooling only)
-  float* slots = nullptr;        // [query groups, H_kv, max_total_rows] (only when a KV head has more than 256 query rows)
+  float* slots = nullptr;        // [query groups, H_kv, max_total_rows] (sized for groups of 256 query rows; used when sweep 2 has more than one group)
   long long wait_limit = 0;      // cycles a device-side wait may take (0: the default, about a second)
   int32_t* idx = nullptr;        // [H_kv, max_total_rows]
   // staging for the host-buffer entry points (allocated on first use): two sets, so that the copies of one

@@ -25,7 +25,8 @@
 // (dapq_score) are exact in bf16 already: the same kernels then run bf16 x bf16 with no conversion.
 //
 // Work decomposition.  CTA = (chunk of K tiles, query group, KV head), one CTA per SM.  A KV head
-// with more than 256 query rows is cut into equal groups; the CTAs of one chunk sit side by side in
+// with more than 256 query rows is cut into equal groups (of up to 256 rows in sweep 1, up to 512 in sweep 2,
+// where a CTA runs two jobs per K tile); the CTAs of one chunk sit side by side in
 // the grid, run at the same time and share their K tiles through L2, so K crosses DRAM once per
 // sweep whatever G*N is.  Each CTA keeps its group resident in shared memory beside a ring of K
 // stages.  23 warps: warp 0 issues the TMA loads, warp 1 the MMAs (and owns tensor memory), warps

@@ -2,8 +2,8 @@
 // summed over the N pseudo queries and the G query heads of the KV head's group.
 //
 //   D[key, query] = K_tile Q_grp^T, keys on tensor-memory lanes, up to 256 query columns.
-// CTA = (chunk of K tiles, query group, KV head): a KV head with more than 256 query rows is cut into
-// groups of equal size, each scored by a CTA of its own against the same K chunk (the CTAs of a chunk
+// CTA = (chunk of K tiles, query group, KV head): a KV head with more than 512 query rows is cut into
+// groups of equal size (a CTA keeps up to 512 rows resident and then runs two jobs per K tile), each scored by a CTA of its own against the same K chunk (the CTAs of a chunk
 // are neighbours in the grid, run at the same time and find each other's K tiles in L2, so K crosses
 // DRAM once); the groups' scores go to separate slots that a small kernel sums in fixed order.
 // A job is one [128 keys x <= 256 queries] accumulator (two fit; four of 128 columns for small groups).
