@@ -693,6 +693,16 @@ def test_evict_random_shapes(dq, dtype, hq, hkv, n, lens, keep):
     _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
 
 
+@pytest.mark.parametrize("hq,n", [(3, 100), (5, 104), (7, 64), (6, 128)])
+def test_evict_more_than_256_query_rows_per_kv_head(dq, hq, n):
+    """300, 520, 448 and 768 query rows on one KV head: sweep 1 cuts them into groups of up to 256 rows, sweep 2
+    into groups of up to 512 whose second job is 48, 16, 192 or 128 columns wide (default fp16 queries)."""
+    w = _small(lens=(900, 130, 1), keep=(90, 130, 1), dtype="bf16", n_q_heads=hq, n_kv_heads=1, n_pseudo=n, n_needles=0,
+               outlier_channels=2)
+    data = gi.draw_layer(w, 0, "cpu")
+    _check_evict(w, data, _gpu_evict(dq, w, data), util.oracle_evict(w, data))
+
+
 def test_evict_largest_batch(dq):
     """DAPQ_MAX_BATCH sequences in one call (1 to 300 tokens each, some keeping every row)."""
     rng = np.random.default_rng(77)
